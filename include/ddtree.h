@@ -1,0 +1,176 @@
+/*
+ * ddtree.h -- C ABI of the DDTree per-round hot path for NVIDIA B200 (sm_100a).
+ *
+ * One speculative-decoding round of DDTree (paper Section 4.1, steps 2-4) between the
+ * drafter's logits and the next bonus token:
+ *
+ *   ddtree_build           step 2 + the "compile" half of step 3: per-position log-softmax and
+ *                          top-K (Sections 3 and 4.3), best-first selection of at most B prefixes
+ *                          (Algorithm 1), flattening into verifier inputs (Section 4.4).
+ *   ddtree_tree_attention  the attention of step 3: every tree row attends to the KV-cache prefix
+ *                          and, inside the tree, to the root, its ancestors and itself (Section 4.4).
+ *   ddtree_accept          step 4: greedy target choice at every row and the verifier walk
+ *                          (Section 4.4, Figure 2(b)).
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its name ends in _host.  The caller owns every
+ *     buffer, including the workspace; the library allocates no device memory in these calls and
+ *     keeps no per-call state.  Buffers of one call must not overlap.
+ *   - Every call validates its arguments on the host, ENQUEUES kernels on `cuda_stream`
+ *     (a cudaStream_t; NULL = the legacy default stream) and returns.  Outputs are valid once
+ *     the stream has been synchronised.  Nothing is launched when a call returns an error.
+ *   - Return value: DDTREE_OK (0) or a positive ddtree_status.  ddtree_last_error() gives a
+ *     thread-local message for the last failing call on the calling thread.
+ *   - Conditions found on the device are data, not errors: when Algorithm 1's heap runs empty
+ *     before B pops, n_rows < B+1 and the remaining rows are padding.
+ *   - Shapes: R requests; L draft positions; V vocabulary; K tokens kept per position; B node
+ *     budget (the root -- the bonus token b -- is not counted, Section 4.2), so a request has
+ *     at most N = B+1 rows, row 0 being the root; W = ceil(N/32) mask words per row.
+ *   - Limits: 1 <= K <= 32, K <= V, 1 <= L <= 32, 1 <= B <= 1024 (the largest budget the paper
+ *     uses, Appendix B), V < 2^31.  Logits must be finite (the paper assumes q_i(v) in (0,1)).
+ *   - Rows of logits must start on 16-byte boundaries (base pointer and row stride); V itself
+ *     may be any size, a ragged tail is read element-wise.
+ *   - Calls are re-entrant; the only hidden state is a per-process cache of device properties
+ *     and TMA descriptors behind a mutex.
+ */
+#ifndef DDTREE_H_
+#define DDTREE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DDTREE_OK = 0,
+    DDTREE_ERR_INVALID_ARG = 1, /* null required pointer, size out of range, misaligned rows    */
+    DDTREE_ERR_UNSUPPORTED = 2, /* valid request this build has no kernel for (e.g. head_dim)   */
+    DDTREE_ERR_WORKSPACE = 3,   /* workspace smaller than the *_workspace_bytes() answer         */
+    DDTREE_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; see ddtree_last_error()    */
+    DDTREE_ERR_DEVICE_TIMEOUT = 5 /* a bounded device-side wait gave up (read via ddtree_device_status) */
+} ddtree_status;
+
+typedef enum { DDTREE_F32 = 0, DDTREE_BF16 = 1 } ddtree_dtype;
+
+/* Static, never-freed strings. */
+const char* ddtree_status_string(int status);
+const char* ddtree_last_error(void);
+
+/* ------------------------------------------------------------------------------------------
+ * ddtree_build -- Sections 3, 4.3 (Algorithm 1) and 4.4 ("flatten ... position ids ... tree
+ * attention" inputs).
+ *
+ * For every request r and draft position i = 1..L, reads the logit row l_i (row r*L + i-1 of
+ * `drafter_logits`, V elements of type `dt`, rows `row_stride_elems` apart), forms
+ * log q_i = l_i - logsumexp(l_i) in fp32 and keeps the K most probable tokens ordered by
+ * (logit descending, token id ascending).  It then runs Algorithm 1: a max-heap keyed by
+ * sigma(rho) = sum_i log q_i^(rho_i), started at the tuple (1); each pop adds a node and pushes
+ * its next sibling (rank <= K) and first child (depth < L); it stops after B pops or when the
+ * heap is empty.  The selected prefixes are written in LEVEL ORDER -- sorted by (depth, rank
+ * tuple) -- so that row 0 is the root, parents precede children and siblings are adjacent in
+ * rank order; this order depends only on the node set, not on the pop order.
+ *
+ * Inputs
+ *   drafter_logits  [R*L rows, V]  dt = F32 or BF16
+ *   root_token      [R] int32      bonus token b carried into the round (Section 3)
+ *   prefix_len      [R] int32      tokens already in the KV cache; b sits at this position
+ * Outputs (all [R, B+1] int32 unless noted; rows >= n_rows[r] are padding)
+ *   n_rows          [R]            1 + number of selected nodes
+ *   node_token                     token id per row (row 0 = root_token); padding -1
+ *   node_parent                    parent row (row 0 = -1); padding -1
+ *   node_depth                     depth (row 0 = 0); padding -1
+ *   position_ids                   prefix_len + depth; padding -1
+ *   anc_mask        [R, B+1, W] uint32  bit j of row i set iff row j is i itself or an ancestor
+ *                                  of i (bit j lives in word j/32, bit j%32); padding rows 0
+ *   first_child, child_count       optional (NULL to skip): first child row (-1 if none), #children
+ *   node_logprob    [R, B+1] fp32  optional: sigma of the row's prefix (root 0, padding 0).  fp32
+ *                                  arithmetic: compare with a tolerance, never bit-for-bit
+ *   topk_token      [R, L, K] int32, topk_logprob [R, L, K] fp32   optional: the per-position table
+ *   workspace                      at least ddtree_build_workspace_bytes(...) bytes, 16-byte aligned
+ * ------------------------------------------------------------------------------------------ */
+size_t ddtree_build_workspace_bytes(int R, int L, int V, int K, int B);
+
+int ddtree_build(const void* drafter_logits, int dt, int64_t row_stride_elems,
+                 int R, int L, int V, int K, int B,
+                 const int32_t* root_token, const int32_t* prefix_len,
+                 int32_t* n_rows, int32_t* node_token, int32_t* node_parent, int32_t* node_depth,
+                 int32_t* position_ids, uint32_t* anc_mask,
+                 int32_t* first_child, int32_t* child_count, float* node_logprob,
+                 int32_t* topk_token, float* topk_logprob,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * ddtree_tree_attention -- Section 4.4 (tree attention), Appendix B (scaled-dot-product
+ * attention with an explicit tree mask is what the paper runs).
+ *
+ * For request r, row i < n_rows[r] and query head h (KV head h / (Hq/Hkv)):
+ *   keys/values = the request's P_r cached rows (all visible) followed by the tree rows j whose
+ *   bit is set in anc_mask[r, i];  out = softmax(q . k * softmax_scale) @ v.
+ * The cache is packed: request r owns rows cu_prefix[r] .. cu_prefix[r+1]-1.
+ *
+ * Inputs
+ *   q                [R, B+1, Hq, d]
+ *   k_cache, v_cache [sum P, Hkv, d]      d contiguous
+ *   cu_prefix_host   [R+1] int32 HOST     exclusive prefix sums of the P_r (used for planning)
+ *   cu_prefix        [R+1] int32 device   the same values on the device
+ *   k_tree, v_tree   [R, B+1, Hkv, d]     this round's K/V of the tree rows (not yet in the cache)
+ *   anc_mask         [R, B+1, W] uint32, n_rows [R] int32   as written by ddtree_build
+ * Outputs
+ *   out              [R, B+1, Hq, d]      same element type as q; rows >= n_rows[r] are left untouched
+ *   lse_or_null      [R, B+1, Hq] fp32    optional natural-log sum of exp(scaled scores)
+ * dt = DDTREE_BF16: bf16 inputs, fp32 accumulation on the tensor cores, probabilities rounded to
+ *   bf16 before the PV product; requires d == 128.  dt = DDTREE_F32: fp32 FMA arithmetic; d in
+ *   {64, 128}.  Hq must be a multiple of Hkv with Hq/Hkv in {1, 2, 4, 8, 16}.
+ * softmax_scale 0 means 1/sqrt(d).  All tensors must be 16-byte aligned.
+ * workspace: at least ddtree_tree_attention_workspace_bytes(...) bytes, 16-byte aligned.
+ * ------------------------------------------------------------------------------------------ */
+size_t ddtree_tree_attention_workspace_bytes(int R, int B, int Hq, int Hkv, int d, int dt,
+                                             const int32_t* cu_prefix_host);
+
+int ddtree_tree_attention(const void* q, const void* k_cache, const void* v_cache,
+                          const int32_t* cu_prefix_host, const int32_t* cu_prefix,
+                          const void* k_tree, const void* v_tree,
+                          const uint32_t* anc_mask, const int32_t* n_rows,
+                          void* out, float* lse_or_null,
+                          int dt, int R, int B, int Hq, int Hkv, int d, float softmax_scale,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * ddtree_accept -- Section 4.4, Figure 2(b) (verifier walk under the greedy decoding rule).
+ *
+ * node_argmax[r, i] = smallest token id attaining the maximum of target logit row r*(B+1)+i.
+ * Walk: cur = 0; while some child c of cur has node_token[c] == node_argmax[cur]: accept c,
+ * cur = c.  bonus_token = node_argmax[cur] (the first unmatched target token, next round's root).
+ *
+ * Inputs
+ *   target_logits [R*(B+1) rows, V]   dt = F32 or BF16; rows >= n_rows[r] are never read
+ *   node_token, node_parent [R, B+1], n_rows [R]   as written by ddtree_build (any order with
+ *                                     parent row < child row is accepted)
+ * Outputs
+ *   accept_len    [R]      number of accepted DRAFTED nodes, 0..L (the bonus token is not counted;
+ *                          tokens committed this round = accept_len + 1)
+ *   accept_nodes  [R, L]   rows of the accepted path in order, -1 padded
+ *   accept_tokens [R, L]   their tokens, -1 padded
+ *   bonus_token   [R]
+ *   node_argmax   [R, B+1] optional; padding rows -1
+ * ------------------------------------------------------------------------------------------ */
+size_t ddtree_accept_workspace_bytes(int R, int B, int V);
+
+int ddtree_accept(const void* target_logits, int dt, int64_t row_stride_elems,
+                  int R, int B, int V, int L,
+                  const int32_t* node_token, const int32_t* node_parent, const int32_t* n_rows,
+                  int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
+                  int32_t* bonus_token, int32_t* node_argmax,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Device-side status word of the current device: 0, or DDTREE_ERR_DEVICE_TIMEOUT if a bounded
+ * wait inside a kernel of this library gave up since the last call.  Synchronises the device,
+ * reads and clears the word. */
+int ddtree_device_status(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DDTREE_H_ */

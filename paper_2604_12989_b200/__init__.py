@@ -1,0 +1,200 @@
+"""Python binding of the DDTree B200 library (libddtree.so, C ABI in include/ddtree.h).
+
+The functions here only marshal arguments: they take torch CUDA tensors (device memory and
+streams are PyTorch's), allocate outputs and workspaces, and pass raw pointers to the three
+entry points.  Every step of the round runs in the library's kernels; there is no fallback:
+if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libddtree.so")
+
+DDTREE_F32, DDTREE_BF16 = 0, 1
+
+EXPORTS = (
+    "ddtree_status_string", "ddtree_last_error",
+    "ddtree_build_workspace_bytes", "ddtree_build",
+    "ddtree_tree_attention_workspace_bytes", "ddtree_tree_attention",
+    "ddtree_accept_workspace_bytes", "ddtree_accept",
+    "ddtree_device_status",
+)
+
+_lib = None
+
+
+class DDTreeError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"ddtree status {status}: {message}")
+        self.status = status
+
+
+def lib() -> ctypes.CDLL:
+    """Load libddtree.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2604_12989_b200._build` "
+                               "(or __graft_entry__.build()); there is no fallback path")
+        L = ctypes.CDLL(LIB_PATH)
+        c = ctypes
+        vp, i32, i64, sz, f32 = c.c_void_p, c.c_int, c.c_int64, c.c_size_t, c.c_float
+        L.ddtree_status_string.restype = c.c_char_p
+        L.ddtree_status_string.argtypes = [i32]
+        L.ddtree_last_error.restype = c.c_char_p
+        L.ddtree_last_error.argtypes = []
+        L.ddtree_build_workspace_bytes.restype = sz
+        L.ddtree_build_workspace_bytes.argtypes = [i32] * 5
+        L.ddtree_build.restype = i32
+        L.ddtree_build.argtypes = [vp, i32, i64, i32, i32, i32, i32, i32] + [vp] * 13 + [vp, sz, vp]
+        L.ddtree_tree_attention_workspace_bytes.restype = sz
+        L.ddtree_tree_attention_workspace_bytes.argtypes = [i32] * 6 + [vp]
+        L.ddtree_tree_attention.restype = i32
+        L.ddtree_tree_attention.argtypes = [vp] * 11 + [i32] * 6 + [f32, vp, sz, vp]
+        L.ddtree_accept_workspace_bytes.restype = sz
+        L.ddtree_accept_workspace_bytes.argtypes = [i32] * 3
+        L.ddtree_accept.restype = i32
+        L.ddtree_accept.argtypes = [vp, i32, i64, i32, i32, i32, i32] + [vp] * 8 + [vp, sz, vp]
+        L.ddtree_device_status.restype = i32
+        L.ddtree_device_status.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        raise DDTreeError(rc, lib().ddtree_last_error().decode())
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.float32:
+        return DDTREE_F32
+    if t.dtype == torch.bfloat16:
+        return DDTREE_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _stream(stream=None) -> int:
+    import torch
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+@dataclass
+class Tree:
+    """Outputs of ddtree_build (torch CUDA tensors).  Shapes: [R] or [R, B+1(, W)]."""
+    n_rows: "torch.Tensor"
+    node_token: "torch.Tensor"
+    node_parent: "torch.Tensor"
+    node_depth: "torch.Tensor"
+    position_ids: "torch.Tensor"
+    anc_mask: "torch.Tensor"  # int32 storage of the uint32 words
+    first_child: "torch.Tensor"
+    child_count: "torch.Tensor"
+    node_logprob: "torch.Tensor"
+    topk_token: "torch.Tensor"
+    topk_logprob: "torch.Tensor"
+    B: int
+    L: int
+    K: int
+
+
+def ddtree_build(drafter_logits, K: int, B: int, root_token, prefix_len, workspace=None, out: Optional[Tree] = None,
+                 stream=None) -> Tree:
+    """drafter_logits [R, L, V] (fp32 or bf16, CUDA, last dim contiguous); root_token, prefix_len [R] int32."""
+    import torch
+    R, L, V = drafter_logits.shape
+    assert drafter_logits.is_cuda and drafter_logits.stride(2) == 1 and drafter_logits.stride(0) == L * drafter_logits.stride(1)
+    dev = drafter_logits.device
+    N, W = B + 1, (B + 1 + 31) // 32
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=dev)
+        out = Tree(torch.empty(R, **i32), torch.empty(R, N, **i32), torch.empty(R, N, **i32), torch.empty(R, N, **i32),
+                   torch.empty(R, N, **i32), torch.empty(R, N, W, **i32), torch.empty(R, N, **i32),
+                   torch.empty(R, N, **i32), torch.empty(R, N, dtype=torch.float32, device=dev),
+                   torch.empty(R, L, K, **i32), torch.empty(R, L, K, dtype=torch.float32, device=dev), B, L, K)
+    need = lib().ddtree_build_workspace_bytes(R, L, V, K, B)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    _check(lib().ddtree_build(
+        drafter_logits.data_ptr(), _dtype_code(drafter_logits), drafter_logits.stride(1), R, L, V, K, B,
+        root_token.data_ptr(), prefix_len.data_ptr(), out.n_rows.data_ptr(), out.node_token.data_ptr(),
+        out.node_parent.data_ptr(), out.node_depth.data_ptr(), out.position_ids.data_ptr(), out.anc_mask.data_ptr(),
+        _ptr(out.first_child), _ptr(out.child_count), _ptr(out.node_logprob), _ptr(out.topk_token),
+        _ptr(out.topk_logprob), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return out
+
+
+def tree_attention_workspace_bytes(R, B, Hq, Hkv, d, dtype_code, cu_prefix_host) -> int:
+    arr = (ctypes.c_int32 * (R + 1))(*[int(x) for x in cu_prefix_host])
+    return lib().ddtree_tree_attention_workspace_bytes(R, B, Hq, Hkv, d, dtype_code, ctypes.addressof(arr))
+
+
+def ddtree_tree_attention(q, k_cache, v_cache, cu_prefix_host, cu_prefix, k_tree, v_tree, anc_mask, n_rows,
+                          out=None, lse=None, softmax_scale: float = 0.0, workspace=None, stream=None):
+    """q [R, B+1, Hq, d]; k_cache/v_cache [sum P, Hkv, d]; k_tree/v_tree [R, B+1, Hkv, d];
+    cu_prefix_host: sequence of R+1 ints (host); cu_prefix: int32 CUDA tensor with the same values.
+    Returns `out` ([R, B+1, Hq, d], same dtype as q; padding rows untouched)."""
+    import torch
+    R, N, Hq, d = q.shape
+    Hkv = k_tree.shape[2]
+    B = N - 1
+    for t in (q, k_cache, v_cache, k_tree, v_tree):
+        assert t.is_cuda and t.is_contiguous() and t.dtype == q.dtype
+    if out is None:
+        out = torch.zeros_like(q)
+    code = _dtype_code(q)
+    arr = (ctypes.c_int32 * (R + 1))(*[int(x) for x in cu_prefix_host])
+    if workspace is None:
+        need = lib().ddtree_tree_attention_workspace_bytes(R, B, Hq, Hkv, d, code, ctypes.addressof(arr))
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+    _check(lib().ddtree_tree_attention(
+        q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), ctypes.addressof(arr), cu_prefix.data_ptr(),
+        k_tree.data_ptr(), v_tree.data_ptr(), anc_mask.data_ptr(), n_rows.data_ptr(), out.data_ptr(), _ptr(lse),
+        code, R, B, Hq, Hkv, d, float(softmax_scale), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return out
+
+
+@dataclass
+class Acceptance:
+    accept_len: "torch.Tensor"  # [R]
+    accept_nodes: "torch.Tensor"  # [R, L]
+    accept_tokens: "torch.Tensor"  # [R, L]
+    bonus_token: "torch.Tensor"  # [R]
+    node_argmax: "torch.Tensor"  # [R, B+1]
+
+
+def ddtree_accept(target_logits, L: int, node_token, node_parent, n_rows, workspace=None,
+                  out: Optional[Acceptance] = None, stream=None) -> Acceptance:
+    """target_logits [R, B+1, V] (fp32 or bf16, CUDA)."""
+    import torch
+    R, N, V = target_logits.shape
+    B = N - 1
+    assert target_logits.is_cuda and target_logits.stride(2) == 1 and target_logits.stride(0) == N * target_logits.stride(1)
+    dev = target_logits.device
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=dev)
+        out = Acceptance(torch.empty(R, **i32), torch.empty(R, L, **i32), torch.empty(R, L, **i32),
+                         torch.empty(R, **i32), torch.empty(R, N, **i32))
+    if workspace is None:
+        workspace = torch.empty(max(lib().ddtree_accept_workspace_bytes(R, B, V), 256), dtype=torch.uint8, device=dev)
+    _check(lib().ddtree_accept(
+        target_logits.data_ptr(), _dtype_code(target_logits), target_logits.stride(1), R, B, V, L,
+        node_token.data_ptr(), node_parent.data_ptr(), n_rows.data_ptr(), out.accept_len.data_ptr(),
+        out.accept_nodes.data_ptr(), out.accept_tokens.data_ptr(), out.bonus_token.data_ptr(),
+        _ptr(out.node_argmax), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return out
+
+
+def device_status() -> None:
+    """Synchronise and raise if a bounded device-side wait gave up since the last call."""
+    _check(lib().ddtree_device_status())

@@ -1,0 +1,79 @@
+// Shared declarations of the DDTree CUDA library (internal; the public surface is include/ddtree.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "ddtree.h"
+
+namespace ddtree {
+
+constexpr int kMaxK = 32;     // tokens kept per position
+constexpr int kMaxL = 32;     // draft positions
+constexpr int kMaxB = 1024;   // node budget
+constexpr int kMaxN = kMaxB + 1;
+
+// Records a message for ddtree_last_error() and returns `code`.
+int fail(int code, const char* fmt, ...);
+
+// Per-row partial of the drafter logits pass over one vocabulary chunk.
+//   m, s: chunk maximum and sum of exp(x - m);  K best (value, id) pairs follow in separate arrays.
+struct BuildPartialLayout {
+    int chunks;        // chunks per row
+    int chunk_elems;   // elements per chunk (multiple of 1024)
+    size_t off_m, off_s, off_val, off_id, total;  // byte offsets into the workspace
+};
+BuildPartialLayout build_partial_layout(int R, int L, int V, int K);
+
+struct ArgmaxLayout {
+    int chunks;
+    int chunk_elems;
+    size_t off_val, off_id, total;
+};
+ArgmaxLayout argmax_layout(int rows, int V);
+
+// Kernel launchers (each enqueues on `st` and returns cudaGetLastError()).
+cudaError_t launch_logits_topk(const void* logits, int dt, int64_t row_stride, int rows, int V, int K,
+                               const BuildPartialLayout& lay, void* ws, cudaStream_t st);
+cudaError_t launch_tree_build(int R, int L, int K, int B, const BuildPartialLayout& lay, const void* ws,
+                              const int32_t* root_token, const int32_t* prefix_len,
+                              int32_t* n_rows, int32_t* node_token, int32_t* node_parent, int32_t* node_depth,
+                              int32_t* position_ids, uint32_t* anc_mask, int32_t* first_child,
+                              int32_t* child_count, float* node_logprob, int32_t* topk_token,
+                              float* topk_logprob, cudaStream_t st);
+cudaError_t launch_row_argmax(const void* logits, int dt, int64_t row_stride, int R, int N, int V,
+                              const int32_t* n_rows, const ArgmaxLayout& lay, void* ws, cudaStream_t st);
+cudaError_t launch_accept_walk(int R, int N, int L, const ArgmaxLayout& lay, const void* ws,
+                               const int32_t* node_token, const int32_t* node_parent, const int32_t* n_rows,
+                               int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
+                               int32_t* bonus_token, int32_t* node_argmax, cudaStream_t st);
+
+struct AttnArgs {
+    const void *q, *k_cache, *v_cache, *k_tree, *v_tree;
+    const int32_t* cu_prefix;
+    const uint32_t* anc_mask;
+    const int32_t* n_rows;
+    void* out;
+    float* lse;
+    int R, B, N, W, Hq, Hkv, G, d;
+    float scale;
+    int max_prefix;     // host-side max over requests of P_r
+    int64_t total_prefix;
+};
+cudaError_t launch_tree_attention_f32(const AttnArgs& a, cudaStream_t st);
+
+size_t tree_attention_bf16_workspace(const AttnArgs& a, const int32_t* cu_prefix_host);
+// Returns a ddtree_status (descriptor creation can fail with its own message).
+int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host, void* ws, size_t ws_bytes,
+                               cudaStream_t st);
+
+// Device status word (bounded waits report here).
+uint32_t* device_status_word();
+
+// ---- small device helpers --------------------------------------------------------------------
+__device__ __forceinline__ bool beats(float v, int id, float w, int jd) {
+    // (value descending, id ascending): does (v,id) rank strictly before (w,jd)?
+    return v > w || (v == w && id < jd);
+}
+
+}  // namespace ddtree

@@ -1,0 +1,58 @@
+"""CPU-only checks of the boundary: the shared library builds, loads without a GPU and exports
+every symbol include/ddtree.h declares; argument validation answers without launching anything."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2604_12989_b200 import _build
+    import paper_2604_12989_b200 as dd
+    _build.build()
+    return dd.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "ddtree.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ddtree_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    import paper_2604_12989_b200 as dd
+    names = declared_symbols()
+    assert len(names) >= 9
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(dd.EXPORTS) == set(names)
+
+
+def test_status_strings(lib):
+    assert lib.ddtree_status_string(0) == b"ok"
+    assert b"workspace" in lib.ddtree_status_string(3)
+
+
+def test_workspace_queries(lib):
+    assert lib.ddtree_build_workspace_bytes(1, 16, 151936, 8, 64) > 0
+    assert lib.ddtree_build_workspace_bytes(1, 16, 151936, 64, 64) == 0  # K > 32
+    assert lib.ddtree_accept_workspace_bytes(16, 128, 151936) > 0
+    cu = (ctypes.c_int32 * 2)(0, 4096)
+    assert lib.ddtree_tree_attention_workspace_bytes(1, 64, 32, 8, 128, 1, ctypes.addressof(cu)) > 0
+    assert lib.ddtree_tree_attention_workspace_bytes(1, 64, 32, 7, 128, 1, ctypes.addressof(cu)) == 0
+
+
+def test_validation_without_gpu(lib):
+    none = [None] * 13
+    assert lib.ddtree_build(None, 0, 0, 1, 1, 1, 1, 1, *none, None, 0, None) == 1
+    assert b"logits is NULL" in lib.ddtree_last_error()
+    buf = ctypes.create_string_buffer(4096)
+    p = (ctypes.addressof(buf) + 15) & ~15
+    assert lib.ddtree_build(p, 0, 8, 1, 1, 8, 9, 1, *none, None, 0, None) == 1  # K > V
+    assert lib.ddtree_build(p, 7, 8, 1, 1, 8, 2, 1, *none, None, 0, None) == 1  # bad dtype
+    assert lib.ddtree_build(p + 4, 0, 8, 1, 1, 8, 2, 1, *none, None, 0, None) == 1  # misaligned
+    assert lib.ddtree_accept(p, 0, 8, 1, 1, 8, 1, *([None] * 8), None, 0, None) == 1  # null outputs
