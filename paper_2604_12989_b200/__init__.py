@@ -113,7 +113,8 @@ def ddtree_build(drafter_logits, K: int, B: int, root_token, prefix_len, workspa
     """drafter_logits [R, L, V] (fp32 or bf16, CUDA, last dim contiguous); root_token, prefix_len [R] int32."""
     import torch
     R, L, V = drafter_logits.shape
-    assert drafter_logits.is_cuda and drafter_logits.stride(2) == 1 and drafter_logits.stride(0) == L * drafter_logits.stride(1)
+    assert drafter_logits.is_cuda and drafter_logits.stride(2) == 1
+    assert R == 1 or drafter_logits.stride(0) == L * drafter_logits.stride(1)
     dev = drafter_logits.device
     N, W = B + 1, (B + 1 + 31) // 32
     if out is None:
@@ -179,7 +180,8 @@ def ddtree_accept(target_logits, L: int, node_token, node_parent, n_rows, worksp
     import torch
     R, N, V = target_logits.shape
     B = N - 1
-    assert target_logits.is_cuda and target_logits.stride(2) == 1 and target_logits.stride(0) == N * target_logits.stride(1)
+    assert target_logits.is_cuda and target_logits.stride(2) == 1
+    assert R == 1 or target_logits.stride(0) == N * target_logits.stride(1)
     dev = target_logits.device
     if out is None:
         i32 = dict(dtype=torch.int32, device=dev)

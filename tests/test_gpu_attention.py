@@ -90,3 +90,77 @@ def test_fp32_padding_rows_untouched_and_no_lse():
     out, _ = gpu_attention(w, att, trees, with_lse=False)
     compare(w, att, trees, out, None)
     assert (out[0, 5:] == 0).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# bf16 (tensor-core path)
+# ---------------------------------------------------------------------------------------------
+
+def bf16_case(R, B, Hq, Hkv, prefix_lens, K=4, L=8, seed=0, sentinel=False):
+    w = wl.small_workload(R=R, L=L, V=600, K=K, B=B, Hq=Hq, Hkv=Hkv, d=128, dtype="bf16",
+                          prefix_lens=prefix_lens, index=40)
+    att, trees = make_case(w, seed=seed)
+    if sentinel:
+        v = np.zeros((R, w.N, Hkv, 128), np.float32)
+        for j in range(w.N):
+            v[:, j, :, j % 128] = 1e3
+        att.v_tree = wl.f32_to_bf16_bits(v)
+    return w, att, trees
+
+
+@pytest.mark.parametrize("P", [0, 1, 7, 127, 128, 129, 300])
+def test_bf16_short_prefixes_and_sentinel_values(P):
+    w, att, trees = bf16_case(2, 70, 8, 2, (P, P + 5 if P else 0), sentinel=True)
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse)
+
+
+@pytest.mark.parametrize("G,Hkv", [(1, 2), (2, 2), (4, 1), (8, 1), (16, 1)])
+def test_bf16_group_sizes(G, Hkv):
+    w, att, trees = bf16_case(1, 40, G * Hkv, Hkv, (200,), seed=G)
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse)
+
+
+def test_bf16_two_tree_tiles_and_heap_that_ran_empty():
+    # B = 200: tree keys span two 128-key tiles; second request has K = 1 chain (n_rows = 9 << B+1)
+    w, att, trees = bf16_case(2, 200, 4, 1, (260, 3), K=4, L=8, seed=3)
+    chain = orc.build(wl.drafter_logits(w, 1, "peak", 3), 1, w.B, 0, 3)
+    trees[1] = chain
+    assert chain.n_rows == 9
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse)
+    assert (out[1, 9:] == 0).all()  # padding rows untouched
+
+
+def test_bf16_many_requests_direct_path_and_repeatability():
+    # R * Hkv * row_tiles >= number of SMs: no KV split, outputs written directly
+    prefix = tuple(int(x) for x in np.random.default_rng(1).integers(1, 400, 40))
+    w, att, trees = bf16_case(40, 31, 16, 4, prefix, seed=5)
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse)
+    out2, lse2 = gpu_attention(w, att, trees)
+    assert np.array_equal(out, out2) and np.array_equal(lse, lse2)
+
+
+def sampled_pairs(w, trees, heads_full, n_random, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for r in range(w.R):
+        n = trees[r].n_rows
+        pairs = [(i, h) for h in heads_full for i in range(n)]
+        pairs += [(int(rng.integers(0, n)), int(rng.integers(0, w.Hq))) for _ in range(n_random)]
+        out.append(pairs)
+    return out
+
+
+@pytest.mark.parametrize("cfg,heads_full,n_random", [(1, tuple(range(32)), 0), (2, (0, 13), 32), (3, (5,), 16),
+                                                      (4, (63,), 48)])
+def test_bf16_full_size_workloads(cfg, heads_full, n_random):
+    """The five workloads at full size in the launch configuration the benchmark times; the oracle
+    evaluates all rows of the named heads plus random (row, head) pairs."""
+    w = wl.WORKLOADS[cfg]
+    att, trees = make_case(w, "peak")
+    out, lse = gpu_attention(w, att, trees)
+    worst = compare(w, att, trees, out, lse, sampled_pairs(w, trees, heads_full, n_random, cfg))
+    print(f"config {cfg}: worst scaled error {worst:.3e}")
