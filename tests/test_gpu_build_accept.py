@@ -157,7 +157,7 @@ def test_forced_acceptance_lengths(want_len):
     free = [v for v in range(w.V) if v not in kid_tokens][:2]
     t[cur, free[0]] = 60.0
     t[cur, free[1]] = 60.0
-    acc = dd.ddtree_accept(torch.from_numpy(t).cuda(), w.L, tree.node_token, tree.node_parent, tree.n_rows)
+    acc = dd.ddtree_accept(torch.from_numpy(t[None]).cuda(), w.L, tree.node_token, tree.node_parent, tree.n_rows)
     torch.cuda.synchronize()
     want = orc.accept_walk(ct.token, ct.parent, ct.n_rows, orc.node_argmax(t))
     assert want.accept_len == len(path) and want.bonus_token == min(free)
