@@ -6,10 +6,15 @@
 // that budget x G rows share each K/V tile and QK^T / PV are dense 128x128x128 contractions.
 //
 // One CTA = one (request, KV head, 128-row tile, KV split).  Warp roles:
-//   warps 0-3  softmax: thread t owns row t (= TMEM lane t): scale, mask, online max/sum, P -> TMEM
-//   warp 4     TMA producer: Q once, then K/V tiles through a 3-stage ring
-//   warp 5     MMA issuer: S = Q K^T (operands in shared memory), O += P V (P read from TMEM,
-//              V as an MN-major shared-memory operand); owns the TMEM allocation
+//   warps 0-7  softmax: two threads per row (TMEM lane = row).  Thread (row, h) owns key columns
+//              [64h, 64h+64) of every KV tile with its OWN reference maximum, sum and O accumulator
+//              (O_0, O_1 in TMEM), so the halves of a row never synchronise inside the loop; at the end
+//              they are merged like two KV splits.  Exponentials (MUFU) are the co-bottleneck of this
+//              kernel, so all eight warps work on every tile
+//   warp 8     TMA producer: Q once, then separate 3-stage rings for K tiles and V tiles
+//   warp 9     MMA issuer: S = Q K^T (operands in shared memory) runs one tile ahead into two TMEM
+//              score buffers; O_h += P_h V_h (P read from TMEM, V as an MN-major shared-memory
+//              operand) as soon as half h of the tile is ready; owns the TMEM allocation
 // The ancestor bitmask is applied only on tree tiles; prefix tiles need at most a length test on
 // the request's last tile.  Each split writes un-normalised fp32 partials; a combine kernel merges
 // them by log-sum-exp.  Every wait is bounded: when one gives up, the CTA raises a flag in the
@@ -26,17 +31,21 @@ namespace {
 
 constexpr int kTile = 128;            // rows per CTA, keys per KV tile, head dim
 constexpr int kStages = 3;
-constexpr int kSoftmaxThreads = 128;
-constexpr int kThreads = 192;
+constexpr int kSBufs = 2;              // score buffers in TMEM: Q K^T runs one tile ahead of the softmax
+constexpr int kSoftmaxThreads = 256;   // two threads per row, 64 key columns each
+constexpr int kGroupThreads = 128;     // threads of one column half
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 320;          // warps 0-7: softmax; 8: TMA producer; 9: MMA issuer
 constexpr uint32_t kHalfBytes = 128 * 64 * 2;      // one 64-wide half of a 128x128 bf16 tile
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;         // S buffers at columns 0 and 128 (P aliases the first 64 of each)
-constexpr uint32_t kColO = 256;
+constexpr uint32_t kColS = 0;         // S buffers at columns 0 and 128; half h's bf16 P overwrites columns [64h, 64h+32)
+constexpr uint32_t kColO = 256;       // O accumulators of the two column halves at columns 256 and 384
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr uint32_t kErrTimeout = 0x5101;
+constexpr uint32_t kErrAlign = 0x5102;
 
 // ---- PTX wrappers --------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -82,28 +91,47 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
-__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
-}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem desc] * B[smem desc]
-__device__ __forceinline__ void umma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+// One lane of a converged warp (all 32 lanes must call this together).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+        "{\n\t.reg .pred P1;\n\t.reg .b32 r;\n\t"
+        "elect.sync r|P1, 0xffffffff;\n\t"
+        "selp.b32 %0, 1, 0, P1;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc].  The accumulate flag is a template argument and the
+// operands are "base + constant": one thread issues every MMA of the CTA, and anything beyond a
+// handful of scalar instructions per MMA makes that thread, not the tensor pipe, the bottleneck.
+template <bool kAccumulate>
+__device__ __forceinline__ void umma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc) {
+    if (kAccumulate)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d), "l"(a), "l"(b), "r"(idesc) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d), "l"(a), "l"(b), "r"(idesc) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void umma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+template <bool kAccumulate>
+__device__ __forceinline__ void umma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc) {
+    if (kAccumulate)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                     ::"r"(d), "r"(a), "l"(b), "r"(idesc) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                     ::"r"(d), "r"(a), "l"(b), "r"(idesc) : "memory");
 }
 
 #define DDTREE_R32(a, o) \
@@ -152,11 +180,39 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
            (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTile >> 4) << 24);
 }
 
+// Optional timeline instrumentation (compiled in only with -DDDTREE_TRACE; development aid).
+#ifdef DDTREE_TRACE
+__device__ unsigned long long* g_trace = nullptr;
+__device__ __forceinline__ void trace_mark(int idx) {
+    if (g_trace) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        g_trace[cta * 64 + idx] = t;
+    }
+}
+#define TRACE(idx) trace_mark(idx)
+__device__ __forceinline__ void trace_clk(int idx) {
+    if (g_trace) {
+        long long t;
+        asm volatile("mov.u64 %0, %%clock64;" : "=l"(t) :: "memory");
+        const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        g_trace[cta * 64 + idx] = static_cast<unsigned long long>(t);
+    }
+}
+#define TRACE_CLK(idx) trace_clk(idx)
+#else
+#define TRACE(idx) ((void)0)
+#define TRACE_CLK(idx) ((void)0)
+#endif
+
 struct Smem {
     uint8_t q[kTileBytes];
-    uint8_t k[kStages][kTileBytes];
+    uint8_t k[kStages][kTileBytes];   // after the last MMA, k[0..1] double as the 64 KB output staging buffer
     uint8_t v[kStages][kTileBytes];
-    uint64_t q_full, k_full[kStages], v_full[kStages], kv_free[kStages], s_full[2], p_ready[2], o_done;
+    uint64_t q_full, k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
+    uint64_t s_full[kSBufs], p_ready[kSBufs][2], o_done[2], fin[2];
+    float xm[2][kTile], xl[2][kTile]; // [column half][row]: reference maximum and sum, exchanged at the end
     uint32_t tmem_base;
     uint32_t abort;
 };
@@ -168,18 +224,44 @@ struct KernelParams {
     __nv_bfloat16* out;
     float* lse;
     float* part_o;   // [S, R, Hkv, rows_pad, 128]
-    float2* part_ml; // [S, R, Hkv, rows_pad] (scaled max in log2 units, sum)
+    float2* part_ml; // [S, R, Hkv, rows_pad] (reference max in log2 units, sum)
     uint32_t* status;
     int R, N, W, Hq, Hkv, G, splits, rows_pad;
     float scale_log2;
 };
 
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Two non-negative finite floats -> packed bf16 pair (low half = a), rounding to nearest with ties
+// away from zero: add half an ulp of bf16 to the bit pattern, keep the upper 16 bits.  Done with
+// integer adds and one byte permute so that it stays off the conversion/transcendental unit, which
+// the exponentials already saturate.
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    return __byte_perm(__float_as_uint(a) + 0x8000u, __float_as_uint(b) + 0x8000u, 0x7632);
+}
+
+// Replace the scores of invisible keys by -inf: bit c of `word` tells whether key c of this
+// 32-key group is visible to this row.
+__device__ __forceinline__ void mask32(uint32_t (&sv)[64], int o, uint32_t word) {
+#pragma unroll
+    for (int c = 0; c < 32; ++c)
+        if (!((word >> c) & 1u)) sv[o + c] = 0xff800000u;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kc,
                            const __grid_constant__ CUtensorMap map_vc, const __grid_constant__ CUtensorMap map_kt,
                            const __grid_constant__ CUtensorMap map_vt, const KernelParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
+    if (smem_u32(smem_raw) & 1023u) {  // the 128-byte swizzle needs 1024-byte aligned tiles
+        if (threadIdx.x == 0) atomicExch(p.status, kErrAlign);
+        return;
+    }
 
     const int split = blockIdx.x;
     const int kvh = blockIdx.y % p.Hkv, rt = blockIdx.y / p.Hkv;
@@ -194,6 +276,7 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     const int my_tiles = max(0, t_end - t_begin);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) TRACE(0);
     const size_t part_row0 = ((static_cast<size_t>(split) * p.R + r) * p.Hkv + kvh) * p.rows_pad + rt * kTile;
 
     if (my_tiles == 0) {  // this split has nothing to do for this request: publish empty partials
@@ -201,23 +284,60 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         return;
     }
 
-    // ---- set-up -------------------------------------------------------------------------------
-    if (tid == 0) {
+    // ---- set-up: the producer initialises the barriers and starts the first copies at once ----
+    volatile uint32_t* abort_flag = &sm.abort;
+    int k_issued = 0, v_issued = 0;  // tiles whose K / V copies were started (producer lane only)
+    auto tile_row = [&](int j, bool& in_prefix) {
+        const int t = t_begin + j;
+        in_prefix = t < prefix_tiles;
+        return in_prefix ? p0 + t * kTile : r * p.N + (t - prefix_tiles) * kTile;
+    };
+    auto load_k = [&](int j) {
+        bool in_prefix;
+        const int row = tile_row(j, in_prefix), s = j % kStages;
+        mbar_expect_tx(smem_u32(&sm.k_full[s]), kTileBytes);
+        for (int h = 0; h < 2; ++h)
+            tma_load_3d(smem_u32(sm.k[s]) + h * kHalfBytes, in_prefix ? &map_kc : &map_kt, smem_u32(&sm.k_full[s]),
+                        h * 64, kvh, row);
+    };
+    auto load_v = [&](int j) {
+        bool in_prefix;
+        const int row = tile_row(j, in_prefix), s = j % kStages;
+        mbar_expect_tx(smem_u32(&sm.v_full[s]), kTileBytes);
+        for (int h = 0; h < 2; ++h)
+            tma_load_3d(smem_u32(sm.v[s]) + h * kHalfBytes, in_prefix ? &map_vc : &map_vt, smem_u32(&sm.v_full[s]),
+                        h * 64, kvh, row);
+    };
+    if (warp == kProducerWarp && lane == 0) {
         mbar_init(smem_u32(&sm.q_full), 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&sm.k_full[s]), 1);
+            mbar_init(smem_u32(&sm.k_free[s]), 1);
             mbar_init(smem_u32(&sm.v_full[s]), 1);
-            mbar_init(smem_u32(&sm.kv_free[s]), 1);
+            mbar_init(smem_u32(&sm.v_free[s]), 1);
+        }
+        for (int b = 0; b < kSBufs; ++b) {
+            mbar_init(smem_u32(&sm.s_full[b]), 1);
+            mbar_init(smem_u32(&sm.p_ready[b][0]), kGroupThreads);
+            mbar_init(smem_u32(&sm.p_ready[b][1]), kGroupThreads);
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&sm.s_full[b]), 1);
-            mbar_init(smem_u32(&sm.p_ready[b]), kSoftmaxThreads);
+            mbar_init(smem_u32(&sm.o_done[b]), 1);
+            mbar_init(smem_u32(&sm.fin[b]), kSoftmaxThreads);
         }
-        mbar_init(smem_u32(&sm.o_done), 1);
         sm.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const int nodes_per_tile = kTile / p.G;
+        mbar_expect_tx(smem_u32(&sm.q_full), kTileBytes);
+        for (int h = 0; h < 2; ++h)
+            tma_load_4d(smem_u32(sm.q) + h * kHalfBytes, &map_q, smem_u32(&sm.q_full), h * 64, 0, kvh,
+                        r * p.N + rt * nodes_per_tile);
+        // K tiles first (the first MMAs need them), then the V tiles
+        for (; k_issued < my_tiles && k_issued < kStages; ++k_issued) load_k(k_issued);
+        for (; v_issued < my_tiles && v_issued < kStages; ++v_issued) load_v(v_issued);
     }
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
                      "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -226,229 +346,275 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
-    volatile uint32_t* abort_flag = &sm.abort;
-    int issued = 0;  // K/V tiles whose copies were started (producer lane only)
+    if (tid == 0) TRACE(1);
 
-    if (warp == 4) {
-        // ---- TMA producer ---------------------------------------------------------------------
+    if (warp == kProducerWarp) {
+        // ---- TMA producer: K ring (freed when Q K^T has read it) and V ring (freed after P V) ---
         if (lane == 0) {
-            prefetch_tensormap(&map_q);
-            prefetch_tensormap(prefix_tiles ? &map_kc : &map_kt);
-            const int nodes_per_tile = kTile / p.G;
-            mbar_expect_tx(smem_u32(&sm.q_full), kTileBytes);
-            for (int h = 0; h < 2; ++h)
-                tma_load_4d(smem_u32(sm.q) + h * kHalfBytes, &map_q, smem_u32(&sm.q_full), h * 64, 0, kvh,
-                            r * p.N + rt * nodes_per_tile);
-            bool ok = true;
-            for (int j = 0; j < my_tiles && ok; ++j) {
-                const int s = j % kStages, t = t_begin + j;
-                if (j >= kStages) ok = mbar_wait(smem_u32(&sm.kv_free[s]), ((j / kStages) - 1) & 1, abort_flag);
-                if (!ok) break;
-                const bool in_prefix = t < prefix_tiles;
-                const CUtensorMap* mk = in_prefix ? &map_kc : &map_kt;
-                const CUtensorMap* mv = in_prefix ? &map_vc : &map_vt;
-                const int row = in_prefix ? p0 + t * kTile : r * p.N + (t - prefix_tiles) * kTile;
-                mbar_expect_tx(smem_u32(&sm.k_full[s]), kTileBytes);
-                for (int h = 0; h < 2; ++h)
-                    tma_load_3d(smem_u32(sm.k[s]) + h * kHalfBytes, mk, smem_u32(&sm.k_full[s]), h * 64, kvh, row);
-                mbar_expect_tx(smem_u32(&sm.v_full[s]), kTileBytes);
-                for (int h = 0; h < 2; ++h)
-                    tma_load_3d(smem_u32(sm.v[s]) + h * kHalfBytes, mv, smem_u32(&sm.v_full[s]), h * 64, kvh, row);
-                issued = j + 1;
+            while (k_issued < my_tiles || v_issued < my_tiles) {
+                if (k_issued < my_tiles) {
+                    if (!mbar_wait(smem_u32(&sm.k_free[k_issued % kStages]), ((k_issued / kStages) - 1) & 1, abort_flag)) break;
+                    load_k(k_issued++);
+                }
+                if (v_issued < my_tiles && v_issued < k_issued) {
+                    if (!mbar_wait(smem_u32(&sm.v_free[v_issued % kStages]), ((v_issued / kStages) - 1) & 1, abort_flag)) break;
+                    load_v(v_issued++);
+                }
             }
         }
-    } else if (warp == 5) {
-        // ---- MMA issuer -----------------------------------------------------------------------
-        if (lane == 0) {
-            constexpr uint32_t idesc_qk = instr_desc(kTile, false);
-            constexpr uint32_t idesc_pv = instr_desc(kTile, true);
-            bool ok = mbar_wait(smem_u32(&sm.q_full), 0, abort_flag);
-            const uint32_t q_addr = smem_u32(sm.q);
-            for (int j = 0; j <= my_tiles && ok; ++j) {
-                if (j < my_tiles) {  // S[j&1] = Q K_j^T
-                    const int s = j % kStages;
-                    ok = mbar_wait(smem_u32(&sm.k_full[s]), (j / kStages) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t k_addr = smem_u32(sm.k[s]);
-                    const uint32_t d_s = tmem + kColS + (j & 1) * kTile;
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                        umma_ss(d_s, smem_desc(q_addr + off, 16), smem_desc(k_addr + off, 16), idesc_qk, kk > 0);
-                    }
-                    tc_commit(smem_u32(&sm.s_full[j & 1]));
-                }
-                if (j > 0) {  // O += P_{j-1} V_{j-1}
-                    const int i = j - 1, s = i % kStages;
-                    ok = mbar_wait(smem_u32(&sm.p_ready[i & 1]), (i >> 1) & 1, abort_flag) &&
-                         mbar_wait(smem_u32(&sm.v_full[s]), (i / kStages) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t v_addr = smem_u32(sm.v[s]);
-                    const uint32_t a_p = tmem + kColS + (i & 1) * kTile;
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)  // 16 keys per instruction
-                        umma_ts(tmem + kColO, a_p + kk * 8, smem_desc(v_addr + kk * 2048, kHalfBytes), idesc_pv,
-                                (i > 0 || kk > 0));
-                    tc_commit(smem_u32(&sm.kv_free[s]));
-                    tc_commit(smem_u32(&sm.o_done));
-                }
+    } else if (warp == kMmaWarp) {
+        // ---- MMA issuer: the whole warp walks the loop (so that addresses live in uniform
+        //      registers) and one elected lane issues; Q K^T runs kSBufs tiles ahead of the softmax ----
+        constexpr uint32_t idesc_qk = instr_desc(kTile, false);
+        constexpr uint32_t idesc_pv = instr_desc(kTile, true);
+        const uint64_t q_desc = smem_desc(smem_u32(sm.q), 16);
+        const uint64_t k_desc0 = smem_desc(smem_u32(sm.k[0]), 16);
+        const uint64_t v_desc0 = smem_desc(smem_u32(sm.v[0]), kHalfBytes);
+        // S[j % kSBufs] = Q K_j^T: 16 head-dim elements (32 bytes) per instruction; the second 64-wide
+        // half of the tiles sits 16 KB further.  Called by the elected lane only.
+        auto issue_qk = [&](int j) {
+            const int s = j % kStages, b = j % kSBufs;
+            const uint64_t kd = k_desc0 + static_cast<uint64_t>(s) * (kTileBytes >> 4);
+            const uint32_t d_s = tmem + kColS + b * kTile;
+            if (j < 6) TRACE(30 + j);
+            umma_ss<false>(d_s, q_desc, kd, idesc_qk);
+            umma_ss<true>(d_s, q_desc + 2, kd + 2, idesc_qk);
+            umma_ss<true>(d_s, q_desc + 4, kd + 4, idesc_qk);
+            umma_ss<true>(d_s, q_desc + 6, kd + 6, idesc_qk);
+            umma_ss<true>(d_s, q_desc + 1024, kd + 1024, idesc_qk);
+            umma_ss<true>(d_s, q_desc + 1026, kd + 1026, idesc_qk);
+            umma_ss<true>(d_s, q_desc + 1028, kd + 1028, idesc_qk);
+            umma_ss<true>(d_s, q_desc + 1030, kd + 1030, idesc_qk);
+            tc_commit(smem_u32(&sm.k_free[s]));
+            tc_commit(smem_u32(&sm.s_full[b]));
+        };
+        auto wait_k = [&](int j) {
+            return __all_sync(kFull, mbar_wait(smem_u32(&sm.k_full[j % kStages]), (j / kStages) & 1, abort_flag));
+        };
+        bool ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.q_full), 0, abort_flag));
+        if (lane == 0) TRACE(2);
+        for (int j = 0; j < my_tiles && j < kSBufs && ok; ++j) {
+            ok = wait_k(j);
+            if (!ok) break;
+            tc_fence_after();
+            if (elect_one()) issue_qk(j);
+            __syncwarp();
+        }
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            // One burst per tile: O_h += P_h V_h for both column halves of tile j, then the scores of
+            // tile j+2 into the S buffer those P halves sat in.  The tensor pipe pays a start-up
+            // latency of a few hundred cycles whenever it has drained, so bursts are kept long.
+            const int s = j % kStages, b = j % kSBufs;
+            const bool more = j + kSBufs < my_tiles;
+            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.v_full[s]), (j / kStages) & 1, abort_flag)) &&
+                 (!more || wait_k(j + kSBufs)) &&
+                 __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[b][0]), (j / kSBufs) & 1, abort_flag)) &&
+                 __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[b][1]), (j / kSBufs) & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t vd = v_desc0 + static_cast<uint64_t>(s) * (kTileBytes >> 4);
+            const uint32_t a_p = tmem + kColS + b * kTile;  // bf16 P: half h in columns [64h, 64h+32)
+            if (elect_one()) {
+                if (j < 5) TRACE(36 + 2 * j);
+                // 16 keys (16 rows of 128 bytes) per instruction; half h covers keys [64h, 64h+64) of the tile
+                if (j > 0) umma_ts<true>(tmem + kColO, a_p, vd, idesc_pv);
+                else umma_ts<false>(tmem + kColO, a_p, vd, idesc_pv);
+                umma_ts<true>(tmem + kColO, a_p + 8, vd + 128, idesc_pv);
+                umma_ts<true>(tmem + kColO, a_p + 16, vd + 256, idesc_pv);
+                umma_ts<true>(tmem + kColO, a_p + 24, vd + 384, idesc_pv);
+                tc_commit(smem_u32(&sm.o_done[0]));
+                if (j > 0) umma_ts<true>(tmem + kColO + kTile, a_p + 64, vd + 512, idesc_pv);
+                else umma_ts<false>(tmem + kColO + kTile, a_p + 64, vd + 512, idesc_pv);
+                umma_ts<true>(tmem + kColO + kTile, a_p + 72, vd + 640, idesc_pv);
+                umma_ts<true>(tmem + kColO + kTile, a_p + 80, vd + 768, idesc_pv);
+                umma_ts<true>(tmem + kColO + kTile, a_p + 88, vd + 896, idesc_pv);
+                tc_commit(smem_u32(&sm.o_done[1]));
+                tc_commit(smem_u32(&sm.v_free[s]));
+                if (more) issue_qk(j + kSBufs);
             }
+            __syncwarp();
         }
     } else {
-        // ---- softmax warps: thread `tid` owns row `tid` of the tile ---------------------------
-        const int grow = rt * kTile + tid;          // row among this KV head's rows
-        const int node = grow / p.G, g = grow % p.G;
+        // ---- softmax: 256 threads; thread (wt, half) owns key columns [64*half, 64*half+64) of row wt in
+        //      every tile, with its own reference maximum, sum and O accumulator: the two halves of a
+        //      row never talk until the end, where they are merged like two KV splits -----------------
+        const int half = tid >> 7, wt = tid & (kTile - 1);
+        const int grow = rt * kTile + wt;           // row among this KV head's rows
+        const int node = grow / p.G;
         const bool valid = node < n;
         const uint32_t* mrow = p.anc_mask + (static_cast<size_t>(r) * p.N + (valid ? node : 0)) * p.W;
-        const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
-        float m_run = -CUDART_INF_F;   // running maximum, in scaled log2 units
+        const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const uint32_t o_addr = lane_addr + kColO + half * kTile;
+        float m_run = -CUDART_INF_F;   // reference maximum of the exponentials, scaled log2 units
         float l_run = 0.f;
         bool ok = true;
         for (int j = 0; j < my_tiles && ok; ++j) {
-            const int t = t_begin + j;
-            const uint32_t s_addr = lane_addr + kColS + (j & 1) * kTile;
-            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.s_full[j & 1]), (j >> 1) & 1, abort_flag));
+            const int t = t_begin + j, b = j % kSBufs;
+            const uint32_t s_addr = lane_addr + kColS + b * kTile + half * 64;
+            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.s_full[b]), (j / kSBufs) & 1, abort_flag));
             if (!ok) break;  // warp-uniform: the TMEM loads/stores below need the whole warp
+            if (wt == 0 && j < 5) TRACE(half ? 20 + 2 * j : 4 + 3 * j);
             tc_fence_after();
-            uint32_t sv[128];
+            uint32_t sv[64];
             TMEM_LD32(sv, 0, s_addr);
             TMEM_LD32(sv, 32, s_addr + 32);
-            TMEM_LD32(sv, 64, s_addr + 64);
-            TMEM_LD32(sv, 96, s_addr + 96);
-            tmem_wait_ld();
 
-            // visibility of the 128 keys of this tile for this row
-            uint32_t vis[4] = {kFull, kFull, kFull, kFull};
+            // visibility of this thread's 64 keys
+            uint32_t vis0 = kFull, vis1 = kFull;
             bool all_visible = true;
             if (t < prefix_tiles) {
-                const int left = P - t * kTile;  // keys of this request in the tile
-                if (left < kTile) {
+                const int left = P - t * kTile - half * 64;  // keys of this request in my column range
+                if (left < 64) {
                     all_visible = false;
-#pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        const int c = left - w * 32;
-                        vis[w] = c >= 32 ? kFull : (c <= 0 ? 0u : ((1u << c) - 1u));
-                    }
+                    vis0 = left >= 32 ? kFull : (left <= 0 ? 0u : ((1u << left) - 1u));
+                    vis1 = left >= 64 ? kFull : (left <= 32 ? 0u : ((1u << (left - 32)) - 1u));
                 }
             } else {
                 all_visible = false;
-                const int w0 = (t - prefix_tiles) * 4;
-#pragma unroll
-                for (int w = 0; w < 4; ++w) vis[w] = (w0 + w < p.W) ? mrow[w0 + w] : 0u;
+                const int w0 = (t - prefix_tiles) * 4 + half * 2;
+                vis0 = w0 < p.W ? mrow[w0] : 0u;
+                vis1 = w0 + 1 < p.W ? mrow[w0 + 1] : 0u;
             }
+            tmem_wait_ld();
+            if (!all_visible) { mask32(sv, 0, vis0); mask32(sv, 32, vis1); }
             float mx = -CUDART_INF_F;
-            if (all_visible) {
 #pragma unroll
-                for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
-            } else {
-#pragma unroll
-                for (int c = 0; c < 128; ++c) {
-                    const float x = ((vis[c >> 5] >> (c & 31)) & 1u) ? __uint_as_float(sv[c]) : -CUDART_INF_F;
-                    sv[c] = __float_as_uint(x);
-                    mx = fmaxf(mx, x);
-                }
-            }
-            const float m_new = fmaxf(m_run, mx * p.scale_log2);
-            const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
-            float rowsum = 0.f;
-            uint32_t pk[64];
-#pragma unroll
-            for (int c = 0; c < 128; c += 2) {
-                const float e0 = exp2f(fmaf(__uint_as_float(sv[c]), p.scale_log2, -m_use));
-                const float e1 = exp2f(fmaf(__uint_as_float(sv[c + 1]), p.scale_log2, -m_use));
-                rowsum += e0 + e1;
-                const __nv_bfloat162 b = __floats2bfloat162_rn(e0, e1);  // low half = even key
-                pk[c >> 1] = *reinterpret_cast<const uint32_t*>(&b);
-            }
-            TMEM_ST32(s_addr, pk, 0);
-            TMEM_ST32(s_addr + 32, pk, 32);
-
-            const float alpha = m_run == -CUDART_INF_F ? 1.f : exp2f(m_run - m_new);
-            l_run = l_run * alpha + rowsum;
-            m_run = m_new;
-            if (j > 0) {
-                // O holds the sum up to tile j-1: wait for that product, then rescale if the maximum moved
-                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done), (j - 1) & 1, abort_flag));
-                if (!ok) break;
-                tc_fence_after();
-                if (__any_sync(kFull, alpha != 1.f)) {
+            for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
+            if (tid == 0 && j < 5) TRACE(5 + 3 * j);
+            // move the reference maximum only when the maximum outgrew it by 2^8: the exponentials
+            // then stay below 2^8 and the O accumulator rarely needs rescaling
+            const float m_tile = mx * p.scale_log2;
+            const bool bump = m_tile > m_run + 8.f;
+            if (__any_sync(kFull, bump)) {
+                const float alpha = bump ? ex2(m_run - m_tile) : 1.f;
+                if (bump) { l_run *= alpha; m_run = m_tile; }
+                if (j > 0) {  // O_half holds the sum over the earlier tiles: wait for it, rescale my row
+                    ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[half]), (j - 1) & 1, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll
                     for (int c0 = 0; c0 < 128; c0 += 32) {
                         uint32_t ov[32];
-                        TMEM_LD32(ov, 0, lane_addr + kColO + c0);
+                        TMEM_LD32(ov, 0, o_addr + c0);
                         tmem_wait_ld();
 #pragma unroll
                         for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
-                        TMEM_ST32(lane_addr + kColO + c0, ov, 0);
+                        TMEM_ST32(o_addr + c0, ov, 0);
                     }
                 }
             }
+            const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
+
+            // exponentials, row sum, bf16 P written over the first 32 of my 64 score columns
+            float rowsum = 0.f;
+            uint32_t pk[32];
+#pragma unroll
+            for (int c = 0; c < 64; c += 2) {
+                const float e0 = ex2(fmaf(__uint_as_float(sv[c]), p.scale_log2, -m_use));
+                const float e1 = ex2(fmaf(__uint_as_float(sv[c + 1]), p.scale_log2, -m_use));
+                rowsum += e0 + e1;
+                pk[c >> 1] = pack_bf16(e0, e1);  // low half = even key
+            }
+            TMEM_ST32(s_addr, pk, 0);
+            l_run += rowsum;
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(smem_u32(&sm.p_ready[j & 1]));
+            mbar_arrive(smem_u32(&sm.p_ready[b][half]));
+            if (wt == 0 && j < 5) TRACE(half ? 21 + 2 * j : 6 + 3 * j);
         }
-        // ---- epilogue ---------------------------------------------------------------------------
-        if (ok) ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done), (my_tiles - 1) & 1, abort_flag));
+
+        // ---- epilogue: merge the two halves, O -> shared memory (swizzled rows) -> coalesced stores --
+        for (int h = 0; h < 2 && ok; ++h)
+            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[h]), (my_tiles - 1) & 1, abort_flag));
+        if (tid == 0) TRACE(46);
+        float4* stage = reinterpret_cast<float4*>(sm.k[0]);  // [128 rows][32 float4], free once all MMAs are done
+        const bool direct = p.splits == 1;
         if (ok) {
             tc_fence_after();
-            const bool direct = p.splits == 1;
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            const size_t orow = ((static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + g) * kTile;
+            sm.xm[half][wt] = m_run;
+            sm.xl[half][wt] = l_run;
+            mbar_arrive(smem_u32(&sm.fin[0]));
+            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.fin[0]), 0, abort_flag));
+        }
+        float l_row = 0.f, m_row = -CUDART_INF_F;
+        if (ok) {
+            const float m_o = sm.xm[half ^ 1][wt], l_o = sm.xl[half ^ 1][wt];
+            m_row = fmaxf(m_run, m_o);
+            const float a_self = m_run == -CUDART_INF_F ? 0.f : ex2(m_run - m_row);
+            const float a_other = m_o == -CUDART_INF_F ? 0.f : ex2(m_o - m_row);
+            l_row = l_run * a_self + l_o * a_other;
+            const float f = direct ? (l_row > 0.f ? 1.f / l_row : 0.f) : 1.f;
+            const float f0 = (half == 0 ? a_self : a_other) * f, f1 = (half == 0 ? a_other : a_self) * f;
+            // this thread merges head-dim columns [64*half, 64*half+64) of its row from both accumulators
 #pragma unroll
-            for (int c0 = 0; c0 < 128; c0 += 32) {
-                uint32_t ov[32];
-                TMEM_LD32(ov, 0, lane_addr + kColO + c0);
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t o0[32], o1[32];
+                TMEM_LD32(o0, 0, lane_addr + kColO + half * 64 + c0);
+                TMEM_LD32(o1, 0, lane_addr + kColO + kTile + half * 64 + c0);
                 tmem_wait_ld();
-                if (direct) {
-                    if (valid) {
-                        uint4* dst = reinterpret_cast<uint4*>(p.out + orow + c0);
 #pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const __nv_bfloat162 b = __floats2bfloat162_rn(
-                                    __uint_as_float(ov[v4 * 8 + 2 * e]) * inv, __uint_as_float(ov[v4 * 8 + 2 * e + 1]) * inv);
-                                w[e] = *reinterpret_cast<const uint32_t*>(&b);
-                            }
-                            dst[v4] = make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    }
-                } else if (valid) {
-                    float4* dst = reinterpret_cast<float4*>(p.part_o + (part_row0 + tid) * kTile + c0);
-#pragma unroll
-                    for (int v4 = 0; v4 < 8; ++v4)
-                        dst[v4] = make_float4(__uint_as_float(ov[v4 * 4]), __uint_as_float(ov[v4 * 4 + 1]),
-                                              __uint_as_float(ov[v4 * 4 + 2]), __uint_as_float(ov[v4 * 4 + 3]));
+                for (int q4 = 0; q4 < 8; ++q4) {
+                    const int g4 = (half * 64 + c0) / 4 + q4;  // float4 group within the row
+                    float4 vv;
+                    vv.x = fmaf(__uint_as_float(o1[q4 * 4]), f1, __uint_as_float(o0[q4 * 4]) * f0);
+                    vv.y = fmaf(__uint_as_float(o1[q4 * 4 + 1]), f1, __uint_as_float(o0[q4 * 4 + 1]) * f0);
+                    vv.z = fmaf(__uint_as_float(o1[q4 * 4 + 2]), f1, __uint_as_float(o0[q4 * 4 + 2]) * f0);
+                    vv.w = fmaf(__uint_as_float(o1[q4 * 4 + 3]), f1, __uint_as_float(o0[q4 * 4 + 3]) * f0);
+                    stage[wt * 32 + (g4 ^ (wt & 31))] = vv;
                 }
             }
+            mbar_arrive(smem_u32(&sm.fin[1]));
+            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.fin[1]), 0, abort_flag));
+        }
+        if (tid == 0) TRACE(47);
+        if (ok) {
+            const int rows_valid = min(kTile, n * p.G - rt * kTile);
             if (direct) {
-                if (valid && p.lse)
-                    p.lse[(static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + g] = (m_run + log2f(l_run)) / kLog2e;
+                // 16 chunks of 8 bf16 per row
+                for (int idx = tid; idx < rows_valid * 16; idx += kSoftmaxThreads) {
+                    const int row = idx >> 4, c8 = idx & 15;
+                    const float4 a = stage[row * 32 + ((2 * c8) ^ (row & 31))];
+                    const float4 bq = stage[row * 32 + ((2 * c8 + 1) ^ (row & 31))];
+                    const __nv_bfloat162 b0 = __floats2bfloat162_rn(a.x, a.y), b1 = __floats2bfloat162_rn(a.z, a.w);
+                    const __nv_bfloat162 b2 = __floats2bfloat162_rn(bq.x, bq.y), b3 = __floats2bfloat162_rn(bq.z, bq.w);
+                    const int gr = rt * kTile + row;
+                    const size_t orow = ((static_cast<size_t>(r) * p.N + gr / p.G) * p.Hq + kvh * p.G + gr % p.G) * kTile;
+                    *reinterpret_cast<uint4*>(p.out + orow + c8 * 8) =
+                        make_uint4(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1),
+                                   *reinterpret_cast<const uint32_t*>(&b2), *reinterpret_cast<const uint32_t*>(&b3));
+                }
+                if (half == 0 && valid && p.lse)
+                    p.lse[(static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + grow % p.G] =
+                        (m_row + log2f(l_row)) / kLog2e;
             } else {
-                p.part_ml[part_row0 + tid] = make_float2(m_run, l_run);
+                float4* dst = reinterpret_cast<float4*>(p.part_o + part_row0 * kTile);
+                for (int idx = tid; idx < rows_valid * 32; idx += kSoftmaxThreads) {
+                    const int row = idx >> 5, g4 = idx & 31;
+                    dst[idx] = stage[row * 32 + (g4 ^ (row & 31))];
+                }
+                if (half == 0) p.part_ml[part_row0 + wt] = make_float2(m_row, l_row);
             }
         }
     }
 
     // ---- teardown -------------------------------------------------------------------------------
+    if (tid == 0) TRACE(48);
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (tid == 0) TRACE(3);
+    if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
     if (sm.abort) {  // CTA-uniform after the barrier above
-        if (warp == 4 && lane == 0) {
+        if (warp == kProducerWarp && lane == 0) {
             // a wait gave up: before the CTA exits, wait (bounded) for every copy still in flight
             uint32_t scratch = 0;
             mbar_wait(smem_u32(&sm.q_full), 0, &scratch);
-            for (int j = max(0, issued - kStages); j < issued; ++j) {
+            for (int j = max(0, k_issued - kStages); j < k_issued; ++j)
                 mbar_wait(smem_u32(&sm.k_full[j % kStages]), (j / kStages) & 1, &scratch);
+            for (int j = max(0, v_issued - kStages); j < v_issued; ++j)
                 mbar_wait(smem_u32(&sm.v_full[j % kStages]), (j / kStages) & 1, &scratch);
-            }
             atomicExch(p.status, kErrTimeout);
         }
         __syncthreads();
@@ -456,7 +622,8 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 }
 
 // Merge the per-split partials of one (request, row, head): out = sum_s w_s O_s / sum_s w_s l_s
-// with w_s = 2^(m_s - max m).
+// with w_s = 2^(m_s - max m).  One warp per output row; lane s first fetches split s's (m, l), so
+// all splits' loads are in flight together (at most 32 splits).
 __global__ void __launch_bounds__(128)
 combine_kernel(const KernelParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -467,19 +634,26 @@ combine_kernel(const KernelParams p) {
     const int r = static_cast<int>(task / (static_cast<long long>(p.Hq) * p.N));
     if (node >= p.n_rows[r]) return;
     const int kvh = h / p.G, grow = node * p.G + h % p.G;
-    float M = -CUDART_INF_F;
-    for (int s = 0; s < p.splits; ++s)
-        M = fmaxf(M, p.part_ml[((static_cast<size_t>(s) * p.R + r) * p.Hkv + kvh) * p.rows_pad + grow].x);
+    const size_t split_stride = static_cast<size_t>(p.R) * p.Hkv * p.rows_pad;
+    const size_t row0 = (static_cast<size_t>(r) * p.Hkv + kvh) * p.rows_pad + grow;
+    float2 ml = make_float2(-CUDART_INF_F, 0.f);
+    if (lane < p.splits) ml = p.part_ml[lane * split_stride + row0];
+    float M = ml.y > 0.f ? ml.x : -CUDART_INF_F;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
+    const float w = ml.y > 0.f ? exp2f(ml.x - M) : 0.f;  // an empty split never wrote its O row
+    float l = w * ml.y;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(kFull, l, o);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    float l = 0.f;
+    const float* po = p.part_o + row0 * kTile + lane * 4;
+#pragma unroll 4
     for (int s = 0; s < p.splits; ++s) {
-        const size_t row = ((static_cast<size_t>(s) * p.R + r) * p.Hkv + kvh) * p.rows_pad + grow;
-        const float2 ml = p.part_ml[row];
-        if (ml.y == 0.f) continue;  // empty split: its O row was never written
-        const float w = exp2f(ml.x - M);
-        l += w * ml.y;
-        const float4 o = *reinterpret_cast<const float4*>(p.part_o + row * kTile + lane * 4);
-        acc[0] += w * o.x; acc[1] += w * o.y; acc[2] += w * o.z; acc[3] += w * o.w;
+        const float ws = __shfl_sync(kFull, w, s);
+        if (ws == 0.f) continue;  // warp-uniform
+        const float4 o = *reinterpret_cast<const float4*>(po + s * split_stride * kTile);
+        acc[0] = fmaf(ws, o.x, acc[0]); acc[1] = fmaf(ws, o.y, acc[1]);
+        acc[2] = fmaf(ws, o.z, acc[2]); acc[3] = fmaf(ws, o.w, acc[3]);
     }
     const float inv = 1.f / l;
     const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv);
@@ -583,6 +757,7 @@ Plan make_plan(const AttnArgs& a) {
         s = 148 / base;
         const int cap = (max_tiles + 1) / 2;  // at least two KV tiles per split
         if (s > cap) s = cap;
+        if (s > 32) s = 32;  // the combine kernel gives one lane to each split
         if (s < 1) s = 1;
     }
     pl.splits = s;
@@ -596,6 +771,13 @@ Plan make_plan(const AttnArgs& a) {
 }  // namespace
 
 size_t tree_attention_bf16_workspace(const AttnArgs& a, const int32_t*) { return make_plan(a).total; }
+
+#ifdef DDTREE_TRACE
+extern "C" int ddtree_debug_set_trace(void* device_buffer) {
+    unsigned long long* ptr = static_cast<unsigned long long*>(device_buffer);
+    return cudaMemcpyToSymbol(g_trace, &ptr, sizeof(ptr)) == cudaSuccess ? 0 : 4;
+}
+#endif
 
 int launch_tree_attention_bf16(const AttnArgs& a, const int32_t*, void* ws, size_t, cudaStream_t st) {
     const Plan pl = make_plan(a);
@@ -623,7 +805,8 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t*, void* ws, size
     p.splits = pl.splits; p.rows_pad = pl.rows_pad;
     p.scale_log2 = a.scale * kLog2e;
 
-    static const size_t smem_bytes = sizeof(Smem) + 1024;
+    static const size_t smem_bytes = sizeof(Smem);
+    static_assert(sizeof(Smem) <= 232448, "exceeds the 227 KB of shared memory a CTA may opt in to");
     {   // opt in to the large dynamic shared-memory size once per device
         static std::mutex mu;
         static bool done[64] = {};
