@@ -89,9 +89,9 @@ int ddtree_build(const void* drafter_logits, int dt, int64_t row_stride_elems, i
     if (workspace_bytes < lay.total)
         return fail(DDTREE_ERR_WORKSPACE, "ddtree_build: workspace %zu < required %zu bytes", workspace_bytes, lay.total);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    cudaError_t e = launch_logits_topk(drafter_logits, dt, row_stride_elems, R * L, V, K, lay, workspace, st);
+    cudaError_t e = launch_logits_stats(drafter_logits, dt, row_stride_elems, R * L, V, lay, workspace, st);
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_build: logits pass: %s", cudaGetErrorString(e));
-    e = launch_tree_build(R, L, K, B, lay, workspace, root_token, prefix_len, n_rows, node_token, node_parent,
+    e = launch_tree_build(R, L, V, K, B, lay, workspace, drafter_logits, dt, row_stride_elems, root_token, prefix_len, n_rows, node_token, node_parent,
                           node_depth, position_ids, anc_mask, first_child, child_count, node_logprob, topk_token,
                           topk_logprob, st);
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_build: tree kernel: %s", cudaGetErrorString(e));

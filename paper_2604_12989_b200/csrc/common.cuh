@@ -16,12 +16,16 @@ constexpr int kMaxN = kMaxB + 1;
 // Records a message for ddtree_last_error() and returns `code`.
 int fail(int code, const char* fmt, ...);
 
-// Per-row partial of the drafter logits pass over one vocabulary chunk.
-//   m, s: chunk maximum and sum of exp(x - m);  K best (value, id) pairs follow in separate arrays.
+// Drafter logits pass: a tile is kTopkChunk consecutive elements of one logits row, reduced by a
+// CTA of kTopkThreads threads; thread t owns the 16-byte vectors v*kTopkThreads + t of the tile.
+// Per tile the pass leaves max and sum of exp(x - max), per warp and per thread the maximum of
+// their elements.
+constexpr int kTopkChunk = 8192;
+constexpr int kTopkThreads = 256;
 struct BuildPartialLayout {
-    int chunks;        // chunks per row
-    int chunk_elems;   // elements per chunk (multiple of 1024)
-    size_t off_m, off_s, off_val, off_id, total;  // byte offsets into the workspace
+    int chunks;        // tiles per row
+    int chunk_elems;   // = kTopkChunk
+    size_t off_m, off_s, off_tmax, off_wmax, total;  // byte offsets into the workspace
 };
 BuildPartialLayout build_partial_layout(int R, int L, int V, int K);
 
@@ -33,9 +37,10 @@ struct ArgmaxLayout {
 ArgmaxLayout argmax_layout(int rows, int V);
 
 // Kernel launchers (each enqueues on `st` and returns cudaGetLastError()).
-cudaError_t launch_logits_topk(const void* logits, int dt, int64_t row_stride, int rows, int V, int K,
-                               const BuildPartialLayout& lay, void* ws, cudaStream_t st);
-cudaError_t launch_tree_build(int R, int L, int K, int B, const BuildPartialLayout& lay, const void* ws,
+cudaError_t launch_logits_stats(const void* logits, int dt, int64_t row_stride, int rows, int V,
+                                const BuildPartialLayout& lay, void* ws, cudaStream_t st);
+cudaError_t launch_tree_build(int R, int L, int V, int K, int B, const BuildPartialLayout& lay, const void* ws,
+                              const void* logits, int dt, int64_t row_stride,
                               const int32_t* root_token, const int32_t* prefix_len,
                               int32_t* n_rows, int32_t* node_token, int32_t* node_parent, int32_t* node_depth,
                               int32_t* position_ids, uint32_t* anc_mask, int32_t* first_child,

@@ -16,6 +16,8 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kUnroll = 4;
+constexpr int kPerThread = kTopkChunk / kThreads;  // elements per thread of a drafter tile (32)
+static_assert(kThreads == kTopkThreads, "tile ownership is defined for 256-thread CTAs");
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr unsigned kFull = 0xffffffffu;
 
@@ -27,6 +29,10 @@ template <> struct Vec16<float> {
         v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
     }
     static __device__ __forceinline__ float scalar(const float* p) { return __ldg(p); }
+    static __device__ __forceinline__ void load_shared(const float* p, float (&v)[4]) {
+        const float4 t = *reinterpret_cast<const float4*>(p);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
 };
 template <> struct Vec16<__nv_bfloat16> {
     static constexpr int N = 8;
@@ -42,49 +48,29 @@ template <> struct Vec16<__nv_bfloat16> {
     static __device__ __forceinline__ float scalar(const __nv_bfloat16* p) {
         return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
     }
-};
-
-// Sorted list of the best entries seen by a warp: lane k holds the k-th best (value, id).
-struct WarpTopK {
-    float tv;   // this lane's entry
-    int ti;
-    float thr_v;  // entry of lane K-1 (what a candidate has to beat)
-    int thr_i;
-    __device__ __forceinline__ void init() { tv = -CUDART_INF_F; ti = -1; thr_v = -CUDART_INF_F; thr_i = -1; }
-    // Warp-collective: insert a candidate that beats the threshold.
-    __device__ __forceinline__ void insert(float v, int id, int K, int lane) {
-        const bool mine_first = beats(tv, ti, v, id);
-        const int pos = __popc(__ballot_sync(kFull, mine_first));
-        const float upv = __shfl_up_sync(kFull, tv, 1);
-        const int upi = __shfl_up_sync(kFull, ti, 1);
-        if (lane == pos) { tv = v; ti = id; }
-        else if (lane > pos) { tv = upv; ti = upi; }
-        thr_v = __shfl_sync(kFull, tv, K - 1);
-        thr_i = __shfl_sync(kFull, ti, K - 1);
-    }
-    // Warp-collective: every lane offers VN candidates vals[e] with ids id0+e.
-    template <int VN>
-    __device__ __forceinline__ void offer(const float (&vals)[VN], int id0, int K, int lane) {
-        unsigned qual = 0;
+    static __device__ __forceinline__ void load_shared(const __nv_bfloat16* p, float (&v)[8]) {
+        const uint4 t = *reinterpret_cast<const uint4*>(p);
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
-        for (int e = 0; e < VN; ++e)
-            if (beats(vals[e], id0 + e, thr_v, thr_i)) qual |= 1u << e;
-        unsigned any = __ballot_sync(kFull, qual != 0);
-        while (any) {
-            const int src = __ffs(any) - 1;
-            any &= any - 1;
-            const unsigned qs = __shfl_sync(kFull, qual, src);
-            const int ids = __shfl_sync(kFull, id0, src);
-#pragma unroll
-            for (int e = 0; e < VN; ++e) {
-                if ((qs >> e) & 1u) {  // warp-uniform
-                    const float v = __shfl_sync(kFull, vals[e], src);
-                    if (beats(v, ids + e, thr_v, thr_i)) insert(v, ids + e, K, lane);
-                }
-            }
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
         }
     }
 };
+
+__device__ __forceinline__ unsigned orderable(float f) {
+    const unsigned u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_orderable(unsigned k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 __device__ __forceinline__ void online_merge(float& m, float& s, float m2, float s2) {
     const float M = fmaxf(m, m2);
@@ -93,97 +79,91 @@ __device__ __forceinline__ void online_merge(float& m, float& s, float m2, float
     m = M;
 }
 
+// Drafter logits pass.  A tile is kTopkChunk consecutive elements of one row; thread t of the CTA
+// owns the 16-byte vectors v*256 + t (v = 0..) of the tile.  The pass is a pure streaming reduction:
+// per tile it writes max and sum of exponentials, per warp the warp's maximum, and per thread the
+// maximum of the thread's 32 elements.  The top-K of a row is recovered afterwards from those thread maxima (tree_build.cu):
+// the K-th largest thread maximum bounds the K-th largest element from below, so only about K
+// threads' elements are ever looked at again.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))),
+                 "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Persistent CTAs walk the tiles.  The next tile streams into shared memory with 16-byte
+// asynchronous copies while the current one is reduced, so the bytes in flight do not depend on
+// how many registers the reduction needs.
 template <typename T>
-__global__ void __launch_bounds__(kThreads)
-logits_topk_kernel(const T* __restrict__ logits, int64_t row_stride, int V, int K, int chunk_elems, int chunks,
-                   float* __restrict__ pm, float* __restrict__ ps, float* __restrict__ pval,
-                   int* __restrict__ pid) {
+__global__ void __launch_bounds__(kThreads, 3)
+logits_stats_kernel(const T* __restrict__ logits, int64_t row_stride, int V, int chunks, int tiles,
+                    float* __restrict__ pm, float* __restrict__ ps, float* __restrict__ tmax,
+                    float* __restrict__ wmax) {
     constexpr int VN = Vec16<T>::N;
-    const int row = blockIdx.x / chunks, chunk = blockIdx.x % chunks;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const T* x = logits + static_cast<int64_t>(row) * row_stride;
-    const int begin = chunk * chunk_elems;
-    const int end = min(V, begin + chunk_elems);
-    const int vec_end = begin + ((end - begin) / VN) * VN;
-
-    WarpTopK top;
-    top.init();
-    float m = -CUDART_INF_F, s = 0.f;
-
-    constexpr int kStep = kThreads * VN;
-    for (int it = begin + warp * 32 * VN; it < vec_end; it += kUnroll * kStep) {
-        float vals[kUnroll][VN];
-        int id0[kUnroll];
-        bool ok[kUnroll];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            id0[u] = it + u * kStep + lane * VN;
-            ok[u] = id0[u] < vec_end;
-            if (ok[u]) Vec16<T>::load(x + id0[u], vals[u]);
-            else {
-#pragma unroll
-                for (int e = 0; e < VN; ++e) vals[u][e] = -CUDART_INF_F;
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            if (it + u * kStep >= vec_end) break;  // warp-uniform
-            if (ok[u]) {
-                float vm = vals[u][0];
-#pragma unroll
-                for (int e = 1; e < VN; ++e) vm = fmaxf(vm, vals[u][e]);
-                if (vm > m) { s *= exp2f((m - vm) * kLog2e); m = vm; }
-#pragma unroll
-                for (int e = 0; e < VN; ++e) s += exp2f((vals[u][e] - m) * kLog2e);
-            }
-            top.offer<VN>(vals[u], id0[u], K, lane);
-        }
-    }
-    // ragged tail of the row (fewer than VN elements), one element per lane of warp 0
-    if (warp == 0 && vec_end < end) {
-        float v1[1];
-        const int id = vec_end + lane;
-        const bool ok = id < end;
-        v1[0] = ok ? Vec16<T>::scalar(x + id) : -CUDART_INF_F;
-        if (ok) {
-            if (v1[0] > m) { s *= exp2f((m - v1[0]) * kLog2e); m = v1[0]; }
-            s += exp2f((v1[0] - m) * kLog2e);
-        }
-        top.offer<1>(v1, id, K, lane);
-    }
-
-    // block-level merge
-    __shared__ float sm_v[kWarps][32];
-    __shared__ int sm_i[kWarps][32];
+    constexpr int NV = kPerThread / VN;
+    extern __shared__ __align__(16) unsigned char topk_smem[];
+    T* buf[2] = {reinterpret_cast<T*>(topk_smem), reinterpret_cast<T*>(topk_smem) + kTopkChunk};
     __shared__ float sm_m[kWarps], sm_s[kWarps];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    auto prefetch = [&](int tile, T* dst) {
+        const int row = tile / chunks, begin = (tile % chunks) * kTopkChunk;
+        const T* x = logits + static_cast<int64_t>(row) * row_stride;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float m2 = __shfl_xor_sync(kFull, m, o);
-        const float s2 = __shfl_xor_sync(kFull, s, o);
-        online_merge(m, s, m2, s2);
-    }
-    sm_v[warp][lane] = lane < K ? top.tv : -CUDART_INF_F;
-    sm_i[warp][lane] = lane < K ? top.ti : -1;
-    if (lane == 0) { sm_m[warp] = m; sm_s[warp] = s; }
-    __syncthreads();
-    if (warp == 0) {
-        for (int w = 1; w < kWarps; ++w) {
-            float v1[1] = {sm_v[w][lane]};
-            // ids are absolute, so offer() is called with a per-lane id and a single element
-            const int id = sm_i[w][lane];
-            unsigned any = __ballot_sync(kFull, beats(v1[0], id, top.thr_v, top.thr_i));
-            while (any) {
-                const int src = __ffs(any) - 1;
-                any &= any - 1;
-                const float v = __shfl_sync(kFull, v1[0], src);
-                const int vi = __shfl_sync(kFull, id, src);
-                if (beats(v, vi, top.thr_v, top.thr_i)) top.insert(v, vi, K, lane);
+        for (int v = 0; v < NV; ++v) {
+            const int off = (v * kThreads + tid) * VN, id0 = begin + off;
+            if (id0 + VN <= V) cp_async16(dst + off, x + id0);
+            else {  // ragged end of the row: element-wise, padded with -inf
+#pragma unroll
+                for (int e = 0; e < VN; ++e) {
+                    if constexpr (sizeof(T) == 4) reinterpret_cast<float*>(dst)[off + e] = id0 + e < V ? Vec16<T>::scalar(x + id0 + e) : -CUDART_INF_F;
+                    else reinterpret_cast<unsigned short*>(dst)[off + e] =
+                        id0 + e < V ? __ldg(reinterpret_cast<const unsigned short*>(x + id0 + e)) : static_cast<unsigned short>(0xff80);
+                }
             }
-            online_merge(m, s, sm_m[w], sm_s[w]);
         }
-        const size_t p = static_cast<size_t>(row) * chunks + chunk;
-        if (lane < K) { pval[p * K + lane] = top.tv; pid[p * K + lane] = top.ti; }
-        if (lane == 0) { pm[p] = m; ps[p] = s; }
+        cp_async_commit();
+    };
+
+    int tile = blockIdx.x;
+    if (tile < tiles) prefetch(tile, buf[0]);
+    for (int it = 0; tile < tiles; tile += gridDim.x, ++it) {
+        const int next = tile + gridDim.x;
+        if (next < tiles) { prefetch(next, buf[(it + 1) & 1]); cp_async_wait<1>(); }
+        else cp_async_wait<0>();
+        __syncthreads();  // the current tile is in shared memory, visible to every thread
+        const T* cur = buf[it & 1];
+        float val[NV][VN];
+#pragma unroll
+        for (int v = 0; v < NV; ++v) Vec16<T>::load_shared(cur + (v * kThreads + tid) * VN, val[v]);
+        float m = -CUDART_INF_F;
+#pragma unroll
+        for (int v = 0; v < NV; ++v)
+#pragma unroll
+            for (int e = 0; e < VN; ++e) m = fmaxf(m, val[v][e]);
+        tmax[static_cast<size_t>(tile) * kThreads + tid] = m;
+        // exponentials relative to the warp maximum, four partial sums to keep the add chain short
+        const float wm = from_orderable(__reduce_max_sync(kFull, orderable(m)));
+        const float mm = wm == -CUDART_INF_F ? 0.f : wm * kLog2e;
+        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int v = 0; v < NV; ++v)
+#pragma unroll
+            for (int e = 0; e < VN; ++e) s4[e & 3] += ex2_approx(fmaf(val[v][e], kLog2e, -mm));
+        float s = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(kFull, s, o);
+        if (lane == 0) { sm_m[warp] = wm; sm_s[warp] = s; wmax[static_cast<size_t>(tile) * kWarps + warp] = wm; }
+        __syncthreads();
+        if (tid == 0) {
+            float M = sm_m[0], S = sm_s[0];
+#pragma unroll
+            for (int w = 1; w < kWarps; ++w) online_merge(M, S, sm_m[w], sm_s[w]);
+            pm[tile] = M;
+            ps[tile] = S;
+        }
+        // the next iteration's first barrier orders these reads before sm_m/sm_s and the buffer are reused
     }
 }
 
@@ -258,16 +238,18 @@ int pick_chunk(int64_t rows, int V, int lo, int hi) {
 }  // namespace
 
 BuildPartialLayout build_partial_layout(int R, int L, int V, int K) {
+    (void)K;
+    (void)pick_chunk;
     BuildPartialLayout lay;
     const int64_t rows = static_cast<int64_t>(R) * L;
-    lay.chunk_elems = pick_chunk(rows, V, 4096, 65536);
+    lay.chunk_elems = kTopkChunk;
     lay.chunks = (V + lay.chunk_elems - 1) / lay.chunk_elems;
     const size_t n = static_cast<size_t>(rows) * lay.chunks;
     lay.off_m = 0;
     lay.off_s = align_up(lay.off_m + n * 4, 256);
-    lay.off_val = align_up(lay.off_s + n * 4, 256);
-    lay.off_id = align_up(lay.off_val + n * K * 4, 256);
-    lay.total = align_up(lay.off_id + n * K * 4, 256);
+    lay.off_tmax = align_up(lay.off_s + n * 4, 256);
+    lay.off_wmax = align_up(lay.off_tmax + n * kThreads * 4, 256);
+    lay.total = align_up(lay.off_wmax + n * kWarps * 4, 256);
     return lay;
 }
 
@@ -282,21 +264,29 @@ ArgmaxLayout argmax_layout(int rows, int V) {
     return lay;
 }
 
-cudaError_t launch_logits_topk(const void* logits, int dt, int64_t row_stride, int rows, int V, int K,
-                               const BuildPartialLayout& lay, void* ws, cudaStream_t st) {
+cudaError_t launch_logits_stats(const void* logits, int dt, int64_t row_stride, int rows, int V,
+                                const BuildPartialLayout& lay, void* ws, cudaStream_t st) {
     char* w = static_cast<char*>(ws);
     float* pm = reinterpret_cast<float*>(w + lay.off_m);
     float* ps = reinterpret_cast<float*>(w + lay.off_s);
-    float* pval = reinterpret_cast<float*>(w + lay.off_val);
-    int* pid = reinterpret_cast<int*>(w + lay.off_id);
-    const unsigned grid = static_cast<unsigned>(lay.chunks) * rows;
-    if (dt == DDTREE_F32)
-        logits_topk_kernel<float><<<grid, kThreads, 0, st>>>(static_cast<const float*>(logits), row_stride, V, K,
-                                                            lay.chunk_elems, lay.chunks, pm, ps, pval, pid);
-    else
-        logits_topk_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(logits),
-                                                                    row_stride, V, K, lay.chunk_elems, lay.chunks,
-                                                                    pm, ps, pval, pid);
+    float* tmax = reinterpret_cast<float*>(w + lay.off_tmax);
+    float* wmax = reinterpret_cast<float*>(w + lay.off_wmax);
+    const int tiles = lay.chunks * rows;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int grid = tiles < sms * 3 ? tiles : sms * 3;  // 3 CTAs per SM fit (2 x 32 KB of staging each)
+    if (dt == DDTREE_F32) {
+        const int smem = 2 * kTopkChunk * 4;
+        cudaError_t e = cudaFuncSetAttribute(logits_stats_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        logits_stats_kernel<float><<<grid, kThreads, smem, st>>>(static_cast<const float*>(logits), row_stride, V,
+                                                                lay.chunks, tiles, pm, ps, tmax, wmax);
+    } else {
+        const int smem = 2 * kTopkChunk * 2;
+        logits_stats_kernel<__nv_bfloat16><<<grid, kThreads, smem, st>>>(static_cast<const __nv_bfloat16*>(logits),
+                                                                        row_stride, V, lay.chunks, tiles, pm, ps, tmax, wmax);
+    }
     return cudaGetLastError();
 }
 

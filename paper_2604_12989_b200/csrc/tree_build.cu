@@ -19,10 +19,63 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kSlots = 1056;  // >= kMaxN, multiple of 32
+constexpr int kMaxHits = 64;
 
 __device__ __forceinline__ unsigned orderable(float f) {
     const unsigned u = __float_as_uint(f);
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Sorted list of the best entries seen by a warp: lane k holds the k-th best (value, id).
+struct WarpTopK {
+    float tv;   // this lane's entry
+    int ti;
+    float thr_v;  // entry of lane K-1 (what a candidate has to beat), never below the floor
+    int thr_i;
+    float floor_v;  // values below the floor are known not to be among the K best
+    __device__ __forceinline__ void init(float floor_value) {
+        tv = -CUDART_INF_F; ti = -1;
+        floor_v = floor_value; thr_v = floor_value; thr_i = 0x7fffffff;
+    }
+    // Warp-collective: insert a candidate that beats the threshold.
+    __device__ __forceinline__ void insert(float v, int id, int K, int lane) {
+        const bool mine_first = beats(tv, ti, v, id);
+        const int pos = __popc(__ballot_sync(kFull, mine_first));
+        const float upv = __shfl_up_sync(kFull, tv, 1);
+        const int upi = __shfl_up_sync(kFull, ti, 1);
+        if (lane == pos) { tv = v; ti = id; }
+        else if (lane > pos) { tv = upv; ti = upi; }
+        thr_v = __shfl_sync(kFull, tv, K - 1);
+        thr_i = __shfl_sync(kFull, ti, K - 1);
+        if (thr_i < 0) { thr_v = floor_v; thr_i = 0x7fffffff; }  // fewer than K entries so far
+    }
+    // Warp-collective: every lane offers VN candidates vals[e] with ids id0+e.
+    template <int VN>
+    __device__ __forceinline__ void offer(const float (&vals)[VN], int id0, int K, int lane) {
+        unsigned qual = 0;
+#pragma unroll
+        for (int e = 0; e < VN; ++e)
+            if (beats(vals[e], id0 + e, thr_v, thr_i)) qual |= 1u << e;
+        unsigned any = __ballot_sync(kFull, qual != 0);
+        while (any) {
+            const int src = __ffs(any) - 1;
+            any &= any - 1;
+            const unsigned qs = __shfl_sync(kFull, qual, src);
+            const int ids = __shfl_sync(kFull, id0, src);
+#pragma unroll
+            for (int e = 0; e < VN; ++e) {
+                if ((qs >> e) & 1u) {  // warp-uniform
+                    const float v = __shfl_sync(kFull, vals[e], src);
+                    if (beats(v, ids + e, thr_v, thr_i)) insert(v, ids + e, K, lane);
+                }
+            }
+        }
+    }
+};
+
+__device__ __forceinline__ float load_logit(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float load_logit(const __nv_bfloat16* p) {
+    return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
 }
 
 __device__ __forceinline__ double warp_sum(double x) {
@@ -30,6 +83,14 @@ __device__ __forceinline__ double warp_sum(double x) {
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(kFull, x, o);
     return x;
 }
+
+#ifdef DDTREE_TRACE
+__device__ long long* g_build_trace = nullptr;
+#define BTRACE(idx) do { if (g_build_trace && blockIdx.x == 0 && threadIdx.x == 0) { long long t_; \
+    asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_) :: "memory"); g_build_trace[idx] = t_; } } while (0)
+#else
+#define BTRACE(idx) ((void)0)
+#endif
 
 struct Shared {
     float logq[kMaxL * kMaxK];
@@ -45,15 +106,18 @@ struct Shared {
     unsigned char depth[kSlots];
     unsigned char rank[kSlots];  // 1-based rank among siblings
     unsigned char cc[kSlots];    // children selected so far
+    int hits[kWarps][kMaxHits];   // per warp: threads of the logits pass whose elements are read again
+    int wlist[kWarps][kMaxHits];  // per warp: warps of the logits pass whose thread maxima are looked at
     int lvl_cnt[kMaxL + 2];
     int lvl_start[kMaxL + 3];
     int lvl_cur[kMaxL + 2];
     int count;
 };
 
+template <typename T>
 __global__ void __launch_bounds__(kThreads)
-tree_build_kernel(int L, int K, int B, int chunks, const float* __restrict__ pm, const float* __restrict__ ps,
-                  const float* __restrict__ pval, const int* __restrict__ pid,
+tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restrict__ pm, const float* __restrict__ ps,
+                  const float* __restrict__ tmax, const float* __restrict__ wmax, const T* __restrict__ logits, int64_t row_stride,
                   const int32_t* __restrict__ root_token, const int32_t* __restrict__ prefix_len,
                   int32_t* __restrict__ n_rows, int32_t* __restrict__ node_token, int32_t* __restrict__ node_parent,
                   int32_t* __restrict__ node_depth, int32_t* __restrict__ position_ids,
@@ -65,6 +129,7 @@ tree_build_kernel(int L, int K, int B, int chunks, const float* __restrict__ pm,
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = B + 1, W = (N + 31) / 32;
 
+    BTRACE(0);
     // ---- 1. merge chunk partials: one warp per draft position ---------------------------------
     for (int i = warp; i < L; i += kWarps) {
         const size_t row = static_cast<size_t>(r) * L + i;
@@ -80,33 +145,88 @@ tree_build_kernel(int L, int K, int B, int chunks, const float* __restrict__ pm,
         S = warp_sum(S);
         const double lse = static_cast<double>(M) + log(S);
 
-        // K best of chunks*K candidates, (value desc, id asc); lane k ends up with rank k+1
-        float tv = -CUDART_INF_F, thr_v = -CUDART_INF_F;
-        int ti = -1, thr_i = -1;
-        const int total = chunks * K;
-        const float* cv = pval + row * total;
-        const int* ci = pid + row * total;
-        for (int j0 = 0; j0 < total; j0 += 32) {
-            const int j = j0 + lane;
-            const float v = j < total ? cv[j] : -CUDART_INF_F;
-            const int id = j < total ? ci[j] : -1;
-            unsigned any = __ballot_sync(kFull, beats(v, id, thr_v, thr_i));
-            while (any) {
-                const int src = __ffs(any) - 1;
-                any &= any - 1;
-                const float sv = __shfl_sync(kFull, v, src);
-                const int si = __shfl_sync(kFull, id, src);
-                if (beats(sv, si, thr_v, thr_i)) {
-                    const int pos = __popc(__ballot_sync(kFull, beats(tv, ti, sv, si)));
-                    const float upv = __shfl_up_sync(kFull, tv, 1);
-                    const int upi = __shfl_up_sync(kFull, ti, 1);
-                    if (lane == pos) { tv = sv; ti = si; }
-                    else if (lane > pos) { tv = upv; ti = upi; }
-                    thr_v = __shfl_sync(kFull, tv, K - 1);
-                    thr_i = __shfl_sync(kFull, ti, K - 1);
+        // K best elements of the row, (value desc, id asc); lane k ends up with rank k+1.
+        // The logits pass left the maximum of every warp's 1024 and every thread's 32 elements.  The
+        // K-th largest of the 32 lane-wise maxima over the warp maxima is reached by at least K warps,
+        // hence by at least K elements: only threads whose maximum reaches it can hold one of the K
+        // best, and there are about K of them.  Their elements are read again and inserted into a
+        // sorted warp list.
+        const int n_w = chunks * (kTopkThreads / 32);
+        const float* wm = wmax + row * n_w;
+        const float* tm = tmax + row * n_w * 32;
+        float lm = -CUDART_INF_F;
+        for (int j = lane; j < n_w; j += 32) lm = fmaxf(lm, wm[j]);
+        float tau;
+        {
+            const unsigned key = orderable(lm);
+            int above = 0;
+#pragma unroll
+            for (int o = 1; o < 32; ++o) above += __shfl_xor_sync(kFull, key, o) > key ? 1 : 0;
+            const unsigned kth = __reduce_min_sync(kFull, above < K ? key : 0xffffffffu);
+            const unsigned u = (kth & 0x80000000u) ? (kth & 0x7fffffffu) : ~kth;
+            tau = fmaxf(__uint_as_float(u), -3.0e38f);  // fewer than K elements in the row: take them all
+        }
+        WarpTopK top;
+        top.init(tau);
+        constexpr int VN = 16 / sizeof(T);               // elements per 16-byte vector
+        constexpr int NV = kTopkChunk / kTopkThreads / VN;  // vectors per thread of a tile
+        const T* x = logits + static_cast<int64_t>(row) * row_stride;
+        int* hits = sh.hits[warp];
+        int n_hits = 0;
+        // up to 4 listed threads per round: lane l fetches vector l%8 of listed thread l/8
+        auto flush = [&]() {
+            for (int h0 = 0; h0 < n_hits; h0 += 4) {
+                const int q = h0 + (lane >> 3), v = lane & 7;
+                float vals[VN];
+#pragma unroll
+                for (int e = 0; e < VN; ++e) vals[e] = -CUDART_INF_F;
+                int id0 = 0;
+                if (q < n_hits && v < NV) {
+                    const int j = hits[q];
+                    id0 = (j / kTopkThreads) * kTopkChunk + (v * kTopkThreads + j % kTopkThreads) * VN;
+#pragma unroll
+                    for (int e = 0; e < VN; ++e)
+                        if (id0 + e < V) vals[e] = load_logit(x + id0 + e);
+                }
+                top.offer<VN>(vals, id0, K, lane);
+            }
+            n_hits = 0;
+        };
+        // threads of listed warps whose maximum reaches tau go to the hit list
+        int* wlist = sh.wlist[warp];
+        int n_wl = 0;
+        auto scan_warps = [&]() {
+            for (int g = 0; g < n_wl; g += 4) {
+                float t4[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) t4[q] = g + q < n_wl ? tm[wlist[g + q] * 32 + lane] : -CUDART_INF_F;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const bool hit = t4[q] >= tau;
+                    const unsigned mask = __ballot_sync(kFull, hit);
+                    if (!mask) continue;
+                    if (n_hits + __popc(mask) > kMaxHits) flush();
+                    if (hit) hits[n_hits + __popc(mask & ((1u << lane) - 1u))] = wlist[g + q] * 32 + lane;
+                    n_hits += __popc(mask);
+                    __syncwarp();
                 }
             }
+            n_wl = 0;
+        };
+        for (int j0 = 0; j0 < n_w; j0 += 32) {
+            const int j = j0 + lane;
+            const bool hit = j < n_w && wm[j] >= tau;
+            const unsigned mask = __ballot_sync(kFull, hit);
+            if (!mask) continue;
+            if (n_wl + __popc(mask) > kMaxHits) scan_warps();
+            if (hit) wlist[n_wl + __popc(mask & ((1u << lane) - 1u))] = j;
+            n_wl += __popc(mask);
+            __syncwarp();
         }
+        scan_warps();
+        flush();
+        const float tv = top.tv;
+        const int ti = top.ti;
         if (lane < K) {
             const float lq = static_cast<float>(static_cast<double>(tv) - lse);
             sh.logq[i * K + lane] = lq;
@@ -116,7 +236,9 @@ tree_build_kernel(int L, int K, int B, int chunks, const float* __restrict__ pm,
         }
     }
     if (tid < kMaxL + 2) { sh.lvl_cnt[tid] = 0; sh.lvl_cur[tid] = 0; }
+    BTRACE(1);
     __syncthreads();
+    BTRACE(2);
 
     // ---- 2. best-first selection (Algorithm 1) on warp 0 ---------------------------------------
     if (warp == 0) {
@@ -164,6 +286,7 @@ tree_build_kernel(int L, int K, int B, int chunks, const float* __restrict__ pm,
             }
         }
         __syncwarp();
+        BTRACE(3);
 
         // ---- 3. level order: rows sorted by (depth, parent row, rank) --------------------------
         for (int j = lane; j < count; j += 32) atomicAdd(&sh.lvl_cnt[sh.depth[j]], 1);
@@ -210,6 +333,7 @@ tree_build_kernel(int L, int K, int B, int chunks, const float* __restrict__ pm,
             __syncwarp();
         }
     }
+    BTRACE(4);
     __syncthreads();
 
     // ---- 4. write the verifier's inputs --------------------------------------------------------
@@ -253,22 +377,40 @@ tree_build_kernel(int L, int K, int B, int chunks, const float* __restrict__ pm,
         }
         anc_mask[o * W + idx] = bits;
     }
+    BTRACE(5);
 }
 
 }  // namespace
 
-cudaError_t launch_tree_build(int R, int L, int K, int B, const BuildPartialLayout& lay, const void* ws,
+#ifdef DDTREE_TRACE
+extern "C" int ddtree_debug_set_build_trace(void* device_buffer) {
+    long long* ptr = static_cast<long long*>(device_buffer);
+    return cudaMemcpyToSymbol(g_build_trace, &ptr, sizeof(ptr)) == cudaSuccess ? 0 : 4;
+}
+#endif
+
+cudaError_t launch_tree_build(int R, int L, int V, int K, int B, const BuildPartialLayout& lay, const void* ws,
+                              const void* logits, int dt, int64_t row_stride,
                               const int32_t* root_token, const int32_t* prefix_len,
                               int32_t* n_rows, int32_t* node_token, int32_t* node_parent, int32_t* node_depth,
                               int32_t* position_ids, uint32_t* anc_mask, int32_t* first_child,
                               int32_t* child_count, float* node_logprob, int32_t* topk_token,
                               float* topk_logprob, cudaStream_t st) {
     const char* w = static_cast<const char*>(ws);
-    tree_build_kernel<<<R, kThreads, 0, st>>>(
-        L, K, B, lay.chunks, reinterpret_cast<const float*>(w + lay.off_m),
-        reinterpret_cast<const float*>(w + lay.off_s), reinterpret_cast<const float*>(w + lay.off_val),
-        reinterpret_cast<const int*>(w + lay.off_id), root_token, prefix_len, n_rows, node_token, node_parent,
-        node_depth, position_ids, anc_mask, first_child, child_count, node_logprob, topk_token, topk_logprob);
+    const float* pm = reinterpret_cast<const float*>(w + lay.off_m);
+    const float* ps = reinterpret_cast<const float*>(w + lay.off_s);
+    const float* tmax = reinterpret_cast<const float*>(w + lay.off_tmax);
+    const float* wmax = reinterpret_cast<const float*>(w + lay.off_wmax);
+    if (dt == DDTREE_F32)
+        tree_build_kernel<float><<<R, kThreads, 0, st>>>(
+            L, V, K, B, lay.chunks, pm, ps, tmax, wmax, static_cast<const float*>(logits), row_stride, root_token, prefix_len,
+            n_rows, node_token, node_parent, node_depth, position_ids, anc_mask, first_child, child_count, node_logprob,
+            topk_token, topk_logprob);
+    else
+        tree_build_kernel<__nv_bfloat16><<<R, kThreads, 0, st>>>(
+            L, V, K, B, lay.chunks, pm, ps, tmax, wmax, static_cast<const __nv_bfloat16*>(logits), row_stride, root_token,
+            prefix_len, n_rows, node_token, node_parent, node_depth, position_ids, anc_mask, first_child, child_count,
+            node_logprob, topk_token, topk_logprob);
     return cudaGetLastError();
 }
 
