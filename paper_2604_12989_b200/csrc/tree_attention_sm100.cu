@@ -485,12 +485,14 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             // then stay below 2^8 and the O accumulator rarely needs rescaling
             const float m_tile = mx * p.scale_log2;
             const bool bump = m_tile > m_run + 8.f;
+            bool saw_o_done = j == 0;  // phase j-1 of o_done must be observed exactly once per tile (see below)
             if (__any_sync(kFull, bump)) {
                 const float alpha = bump ? ex2(m_run - m_tile) : 1.f;
                 if (bump) { l_run *= alpha; m_run = m_tile; }
                 if (j > 0) {  // O_half holds the sum over the earlier tiles: wait for it, rescale my row
                     ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[half]), (j - 1) & 1, abort_flag));
                     if (!ok) break;
+                    saw_o_done = true;
                     tc_fence_after();
 #pragma unroll
                     for (int c0 = 0; c0 < 128; c0 += 32) {
@@ -518,6 +520,13 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             TMEM_ST32(s_addr, pk, 0);
             l_run += rowsum;
             tmem_wait_st();
+            // A parity wait cannot tell phase j-1 from phase j-3: a thread that skipped phases could
+            // sail through a later wait while the product it needs is still running.  So every tile
+            // observes the previous tile's o_done, here at the latest (by now it has long completed).
+            if (!saw_o_done) {
+                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[half]), (j - 1) & 1, abort_flag));
+                if (!ok) break;
+            }
             tc_fence_before();
             mbar_arrive(smem_u32(&sm.p_ready[b][half]));
             if (wt == 0 && j < 5) TRACE(half ? 21 + 2 * j : 6 + 3 * j);

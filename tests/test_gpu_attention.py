@@ -164,3 +164,21 @@ def test_bf16_full_size_workloads(cfg, heads_full, n_random):
     out, lse = gpu_attention(w, att, trees)
     worst = compare(w, att, trees, out, lse, sampled_pairs(w, trees, heads_full, n_random, cfg))
     print(f"config {cfg}: worst scaled error {worst:.3e}")
+
+
+def test_bf16_first_call_of_a_fresh_process():
+    """The first launch of a process runs with cold instruction caches and unusual warp timing; a
+    missed wait inside the kernel shows up there first.  Two-tile, unsplit case in a child process."""
+    import subprocess
+    import sys
+    code = (
+        "import numpy as np\n"
+        "from tests import test_gpu_attention as T\n"
+        "w, att, trees = T.bf16_case(1, 20, 4, 1, (128,))\n"
+        "out, lse = T.gpu_attention(w, att, trees)\n"
+        "T.compare(w, att, trees, out, lse)\n"
+        "print('fresh-process ok')\n")
+    import os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0 and "fresh-process ok" in res.stdout, res.stdout + res.stderr
