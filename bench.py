@@ -34,8 +34,8 @@ METRIC = "ddtree_verify_rounds_per_s"
 UNIT = "rounds/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of tree_attention_bf16_kernel on the
-# benchmark workload, from the ncu capture summarised under profiles/ (None until captured).
-NCU_TRAFFIC_BYTES = {1: None}
+# benchmark workload, from the ncu capture summarised in profiles/tree_attention_bf16_config1.txt.
+NCU_TRAFFIC_BYTES = {1: 17652736}
 
 
 def peaks():
@@ -432,9 +432,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=1, help="workload index (1 = the Qwen3-8B-shaped single request)")
     ap.add_argument("--variant", default="lit", choices=wl.VARIANTS)
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling small cases only)")
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     args = ap.parse_args()
     w = wl.WORKLOADS[args.config]
+    if args.layers > 0:
+        import dataclasses
+        w = dataclasses.replace(w, layers=args.layers)
     if args.impl == "reference":
         run_reference(args, w)
     else:
