@@ -165,6 +165,39 @@ int ddtree_accept(const void* target_logits, int dt, int64_t row_stride_elems,
                   int32_t* bonus_token, int32_t* node_argmax,
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* ------------------------------------------------------------------------------------------
+ * ddtree_accept_static_scratch -- the paper has no counterpart; this is a packaging variant of
+ * ddtree_accept for callers that cannot hand over a workspace.
+ *
+ * Who needs it: code that runs where device memory can no longer be obtained -- a decoding loop
+ * inside a serving engine whose memory pool was carved up at start-up (every byte belongs to the
+ * KV cache or to activations, and cudaMalloc at this point would either fail or stall every
+ * stream of the process while the driver maps memory), a plug-in that is handed tensors but has
+ * no allocator of its own, or a real-time thread that must not enter the driver's allocation
+ * path.  Such a caller still owns its inputs and outputs; what it lacks is a place for the
+ * per-chunk (max, arg-max) partials of the target-logits pass.
+ *
+ * Same arguments, outputs and errors as ddtree_accept without the workspace pair.  The partials
+ * go to a fixed array inside the library (DDTREE_STATIC_SCRATCH_BYTES bytes of device memory per
+ * GPU, held from the moment the library is loaded on that GPU until the process exits).
+ *   - Limit: ddtree_accept_workspace_bytes(R, B, V) must not exceed DDTREE_STATIC_SCRATCH_BYTES;
+ *     larger problems are refused with DDTREE_ERR_WORKSPACE and nothing is launched.
+ *   - The first call on each device looks up the array's device address (one driver query, no
+ *     allocation).  Make that first call outside any stream capture.
+ *   - Every call on a device uses the same array.  Nothing in it has to start at zero (every
+ *     partial that is read was written by the same call), but two calls whose kernels overlap on
+ *     the GPU -- different streams, or different host threads -- overwrite each other's partials:
+ *     serialise them (one stream, or an event between them).
+ *   - The call itself allocates nothing, neither on the device nor through any library.
+ * ------------------------------------------------------------------------------------------ */
+#define DDTREE_STATIC_SCRATCH_BYTES (256u * 1024u)
+
+int ddtree_accept_static_scratch(const void* target_logits, int dt, int64_t row_stride_elems,
+                                 int R, int B, int V, int L,
+                                 const int32_t* node_token, const int32_t* node_parent, const int32_t* n_rows,
+                                 int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
+                                 int32_t* bonus_token, int32_t* node_argmax, void* cuda_stream);
+
 /* Device-side status word of the current device: 0, or DDTREE_ERR_DEVICE_TIMEOUT if a bounded
  * wait inside a kernel of this library gave up since the last call.  Synchronises the device,
  * reads and clears the word. */

@@ -21,7 +21,7 @@ EXPORTS = (
     "ddtree_status_string", "ddtree_last_error",
     "ddtree_build_workspace_bytes", "ddtree_build",
     "ddtree_tree_attention_workspace_bytes", "ddtree_tree_attention",
-    "ddtree_accept_workspace_bytes", "ddtree_accept",
+    "ddtree_accept_workspace_bytes", "ddtree_accept", "ddtree_accept_static_scratch",
     "ddtree_device_status",
 )
 
@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.ddtree_accept_workspace_bytes.argtypes = [i32] * 3
         L.ddtree_accept.restype = i32
         L.ddtree_accept.argtypes = [vp, i32, i64, i32, i32, i32, i32] + [vp] * 8 + [vp, sz, vp]
+        L.ddtree_accept_static_scratch.restype = i32
+        L.ddtree_accept_static_scratch.argtypes = [vp, i32, i64, i32, i32, i32, i32] + [vp] * 8 + [vp]
         L.ddtree_device_status.restype = i32
         L.ddtree_device_status.argtypes = []
         _lib = L
@@ -194,6 +196,26 @@ def ddtree_accept(target_logits, L: int, node_token, node_parent, n_rows, worksp
         node_token.data_ptr(), node_parent.data_ptr(), n_rows.data_ptr(), out.accept_len.data_ptr(),
         out.accept_nodes.data_ptr(), out.accept_tokens.data_ptr(), out.bonus_token.data_ptr(),
         _ptr(out.node_argmax), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return out
+
+
+STATIC_SCRATCH_BYTES = 256 * 1024
+
+
+def ddtree_accept_static_scratch(target_logits, L: int, node_token, node_parent, n_rows, out: Acceptance,
+                                 stream=None) -> Acceptance:
+    """ddtree_accept for callers that cannot provide a workspace: the per-chunk partials go to a
+    fixed array inside the library (STATIC_SCRATCH_BYTES per GPU).  This wrapper allocates nothing
+    either: `out` must be given.  Calls on one device share the array, so do not let two of them
+    overlap on the GPU; make the first call on a device outside any stream capture."""
+    R, N, V = target_logits.shape
+    assert target_logits.is_cuda and target_logits.stride(2) == 1
+    assert R == 1 or target_logits.stride(0) == N * target_logits.stride(1)
+    _check(lib().ddtree_accept_static_scratch(
+        target_logits.data_ptr(), _dtype_code(target_logits), target_logits.stride(1), R, N - 1, V, L,
+        node_token.data_ptr(), node_parent.data_ptr(), n_rows.data_ptr(), out.accept_len.data_ptr(),
+        out.accept_nodes.data_ptr(), out.accept_tokens.data_ptr(), out.bonus_token.data_ptr(),
+        _ptr(out.node_argmax), _stream(stream)))
     return out
 
 

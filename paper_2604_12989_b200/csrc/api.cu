@@ -3,6 +3,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cmath>
+#include <mutex>
 
 namespace ddtree {
 
@@ -200,6 +201,52 @@ int ddtree_tree_attention(const void* q, const void* k_cache, const void* v_cach
     if (workspace_bytes < need)
         return fail(DDTREE_ERR_WORKSPACE, "ddtree_tree_attention: workspace %zu < required %zu bytes", workspace_bytes, need);
     return launch_tree_attention_bf16(a, cu_prefix_host, workspace, workspace_bytes, st);
+}
+
+// Scratch for ddtree_accept_static_scratch: lives in the library image, one copy per GPU that
+// loads it.  Host code must not pass `g_static_scratch` itself to a kernel: in host code that name
+// is only a handle for the runtime; the device address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[DDTREE_STATIC_SCRATCH_BYTES];
+
+// Device address of the scratch array on the current device (looked up once per device).
+static int static_scratch_ptr(void** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void* ptr[kMaxDevices] = {};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_accept_static_scratch: cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices)
+        return fail(DDTREE_ERR_UNSUPPORTED, "ddtree_accept_static_scratch: device index %d out of range", dev);
+    std::lock_guard<std::mutex> g(mu);
+    if (!ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);  // the current device is `dev`
+        if (e != cudaSuccess || !p)
+            return fail(DDTREE_ERR_CUDA, "ddtree_accept_static_scratch: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        ptr[dev] = p;
+    }
+    *out = ptr[dev];
+    return DDTREE_OK;
+}
+
+int ddtree_accept_static_scratch(const void* target_logits, int dt, int64_t row_stride_elems, int R, int B, int V, int L,
+                                 const int32_t* node_token, const int32_t* node_parent, const int32_t* n_rows,
+                                 int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
+                                 int32_t* bonus_token, int32_t* node_argmax, void* cuda_stream) {
+    if (R < 1 || B < 1 || B > kMaxB || V < 1)
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_accept_static_scratch: R, B, V out of range (got %d %d %d)", R, B, V);
+    const size_t need = argmax_layout(R * (B + 1), V).total;
+    if (need > DDTREE_STATIC_SCRATCH_BYTES)
+        return fail(DDTREE_ERR_WORKSPACE,
+                    "ddtree_accept_static_scratch: needs %zu bytes of scratch, the built-in array holds %u; "
+                    "use ddtree_accept with a caller-provided workspace", need, DDTREE_STATIC_SCRATCH_BYTES);
+    void* scratch = nullptr;
+    const int rc = static_scratch_ptr(&scratch);
+    if (rc) return rc;
+    return ddtree_accept(target_logits, dt, row_stride_elems, R, B, V, L, node_token, node_parent, n_rows, accept_len,
+                         accept_nodes, accept_tokens, bonus_token, node_argmax, scratch, DDTREE_STATIC_SCRATCH_BYTES,
+                         cuda_stream);
 }
 
 int ddtree_device_status(void) {
