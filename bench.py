@@ -58,6 +58,23 @@ def attention_work(w: wl.Workload, depths_sum_plus_rows: int):
     return byt, flops
 
 
+def max_over_ranks(value: float, device="cpu") -> float:
+    """Largest `value` over all ranks of the default process group (identity without one)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rounds_per_s(requests_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Every rank runs an independent replica (no data-path collective): the job's throughput is the
+    requests of all ranks over the slowest rank's step time."""
+    return requests_per_rank * world / (ms_per_step * 1e-3)
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -291,11 +308,7 @@ def run_gpu(args, w):
         graph.replay()
     torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
-    ms = torch.tensor([ms_total / args.steps], device=dev, dtype=torch.float64)
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    ms_per_step = float(ms.item())
+    ms_per_step = max_over_ranks(ms_total / args.steps, dev)
     dd.device_status()
 
     # ---- per-call duration of the dominant kernel (tree attention), measured live ----------------
@@ -363,11 +376,7 @@ def run_gpu(args, w):
         accepted = e2e_round()
     e1.record()
     barrier()
-    e2e_ms = torch.tensor([e0.elapsed_time(e1) / args.steps], device=dev, dtype=torch.float64)
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_ms = float(e2e_ms.item())
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1) / args.steps, dev)
 
     if rank != 0:
         return
@@ -395,9 +404,8 @@ def run_gpu(args, w):
     probe_s, _, _ = oracle_round_seconds(w, variant, 8)
     per_pair = probe_s / (w.layers * sum(n_rows) * w.Hq) if probe_s > 0 else 1e-3  # rough cost of one pair
     cpu_s, sample, threads = oracle_round_seconds(w, variant, int(min(max(32, 10.0 / max(per_pair, 1e-5)), 2048)))
-    rounds = w.R * world
     line = {
-        "metric": METRIC, "value": rounds / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": whole_job_rounds_per_s(w.R, world, ms_per_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if bf else "f32", "data": "synthetic",
         "config": {"workload": f"config {w.index} ({w.name})", "variant": variant, "R": w.R, "L": w.L, "V": w.V,
@@ -412,7 +420,7 @@ def run_gpu(args, w):
                      "accept": stage_ms["accept"] * 1e3},
         "logits_pass_GBps": logits_gbs,
         "clocks": clocks,
-        "e2e": {"value": rounds / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+        "e2e": {"value": whole_job_rounds_per_s(w.R, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms, "note": "per round: drafter logits, per-layer Q and tree K/V, target logits "
                 "copied from pinned host memory; accept outputs read back; the KV cache is state and stays in HBM"},
         "gpu_launches": launches_per_round * args.steps,
