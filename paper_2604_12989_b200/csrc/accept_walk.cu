@@ -20,6 +20,7 @@ accept_walk_kernel(int N, int L, int chunks, const float* __restrict__ pval, con
     __shared__ int s_token[kMaxN];
     __shared__ short s_parent[kMaxN];
     const int r = blockIdx.x, tid = threadIdx.x;
+    pdl_wait();
     const int n = min(n_rows[r], N);
     const size_t o = static_cast<size_t>(r) * N;
     for (int row = tid; row < N; row += kThreads) {
@@ -75,11 +76,9 @@ cudaError_t launch_accept_walk(int R, int N, int L, const ArgmaxLayout& lay, con
                                int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
                                int32_t* bonus_token, int32_t* node_argmax, cudaStream_t st) {
     const char* w = static_cast<const char*>(ws);
-    accept_walk_kernel<<<R, kThreads, 0, st>>>(N, L, lay.chunks, reinterpret_cast<const float*>(w + lay.off_val),
-                                               reinterpret_cast<const int*>(w + lay.off_id), node_token,
-                                               node_parent, n_rows, accept_len, accept_nodes, accept_tokens,
-                                               bonus_token, node_argmax);
-    return cudaGetLastError();
+    return launch_pdl(accept_walk_kernel, dim3(R), dim3(kThreads), 0, st, N, L, lay.chunks,
+                      reinterpret_cast<const float*>(w + lay.off_val), reinterpret_cast<const int*>(w + lay.off_id),
+                      node_token, node_parent, n_rows, accept_len, accept_nodes, accept_tokens, bonus_token, node_argmax);
 }
 
 }  // namespace ddtree

@@ -75,6 +75,32 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
 // Device status word (bounded waits report here).
 uint32_t* device_status_word();
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// Every kernel of this library is launched with programmatic stream serialisation: it may be scheduled
+// while the kernel before it in the stream drains, which hides most of the launch latency between the
+// ~76 small kernels of a round.  In exchange every kernel calls pdl_wait() before it touches global
+// memory: that blocks until the preceding kernel has completed and its writes are visible (and is a
+// no-op after a normal launch).  No kernel signals early; measured on B200, explicit early triggers
+// made the captured round slower.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+#endif
+
 // ---- small device helpers --------------------------------------------------------------------
 __device__ __forceinline__ bool beats(float v, int id, float w, int jd) {
     // (value descending, id ascending): does (v,id) rank strictly before (w,jd)?

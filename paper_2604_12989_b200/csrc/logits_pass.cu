@@ -106,6 +106,7 @@ logits_stats_kernel(const T* __restrict__ logits, int64_t row_stride, int V, int
     T* buf[2] = {reinterpret_cast<T*>(topk_smem), reinterpret_cast<T*>(topk_smem) + kTopkChunk};
     __shared__ float sm_m[kWarps], sm_s[kWarps];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_wait();
 
     auto prefetch = [&](int tile, T* dst) {
         const int row = tile / chunks, begin = (tile % chunks) * kTopkChunk;
@@ -172,6 +173,7 @@ __global__ void __launch_bounds__(kThreads)
 row_argmax_kernel(const T* __restrict__ logits, int64_t row_stride, int N, int V, const int32_t* __restrict__ n_rows,
                   int chunk_elems, int chunks, float* __restrict__ pval, int* __restrict__ pid) {
     constexpr int VN = Vec16<T>::N;
+    pdl_wait();
     const int row = blockIdx.x / chunks, chunk = blockIdx.x % chunks;
     if (row % N >= n_rows[row / N]) return;  // padding row: never read
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -280,14 +282,13 @@ cudaError_t launch_logits_stats(const void* logits, int dt, int64_t row_stride, 
         const int smem = 2 * kTopkChunk * 4;
         cudaError_t e = cudaFuncSetAttribute(logits_stats_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        logits_stats_kernel<float><<<grid, kThreads, smem, st>>>(static_cast<const float*>(logits), row_stride, V,
-                                                                lay.chunks, tiles, pm, ps, tmax, wmax);
+        return launch_pdl(logits_stats_kernel<float>, dim3(grid), dim3(kThreads), smem, st,
+                          static_cast<const float*>(logits), row_stride, V, lay.chunks, tiles, pm, ps, tmax, wmax);
     } else {
         const int smem = 2 * kTopkChunk * 2;
-        logits_stats_kernel<__nv_bfloat16><<<grid, kThreads, smem, st>>>(static_cast<const __nv_bfloat16*>(logits),
-                                                                        row_stride, V, lay.chunks, tiles, pm, ps, tmax, wmax);
+        return launch_pdl(logits_stats_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), smem, st,
+                          static_cast<const __nv_bfloat16*>(logits), row_stride, V, lay.chunks, tiles, pm, ps, tmax, wmax);
     }
-    return cudaGetLastError();
 }
 
 cudaError_t launch_row_argmax(const void* logits, int dt, int64_t row_stride, int R, int N, int V,
@@ -297,13 +298,11 @@ cudaError_t launch_row_argmax(const void* logits, int dt, int64_t row_stride, in
     int* pid = reinterpret_cast<int*>(w + lay.off_id);
     const unsigned grid = static_cast<unsigned>(lay.chunks) * R * N;
     if (dt == DDTREE_F32)
-        row_argmax_kernel<float><<<grid, kThreads, 0, st>>>(static_cast<const float*>(logits), row_stride, N, V,
-                                                           n_rows, lay.chunk_elems, lay.chunks, pval, pid);
-    else
-        row_argmax_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(static_cast<const __nv_bfloat16*>(logits),
-                                                                   row_stride, N, V, n_rows, lay.chunk_elems,
-                                                                   lay.chunks, pval, pid);
-    return cudaGetLastError();
+        return launch_pdl(row_argmax_kernel<float>, dim3(grid), dim3(kThreads), 0, st, static_cast<const float*>(logits),
+                          row_stride, N, V, n_rows, lay.chunk_elems, lay.chunks, pval, pid);
+    return launch_pdl(row_argmax_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), 0, st,
+                      static_cast<const __nv_bfloat16*>(logits), row_stride, N, V, n_rows, lay.chunk_elems, lay.chunks,
+                      pval, pid);
 }
 
 }  // namespace ddtree

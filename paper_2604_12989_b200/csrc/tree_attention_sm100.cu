@@ -263,6 +263,7 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         return;
     }
 
+    pdl_wait();               // everything read below may come from the previous kernel of the stream
     const int split = blockIdx.x;
     const int kvh = blockIdx.y % p.Hkv, rt = blockIdx.y / p.Hkv;
     const int r = blockIdx.z;
@@ -636,6 +637,7 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 __global__ void __launch_bounds__(128)
 combine_kernel(const KernelParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_wait();  // the split partials come from the attention kernel launched just before
     const long long task = static_cast<long long>(blockIdx.x) * 4 + warp;
     if (task >= static_cast<long long>(p.R) * p.N * p.Hq) return;
     const int h = static_cast<int>(task % p.Hq);
@@ -832,13 +834,11 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t*, void* ws, size
         }
     }
     dim3 grid(pl.splits, pl.row_tiles * a.Hkv, a.R);
-    tree_attention_bf16_kernel<<<grid, kThreads, smem_bytes, st>>>(mq, mkc, mvc, mkt, mvt, p);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(tree_attention_bf16_kernel, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, p);
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: launch: %s", cudaGetErrorString(e));
     if (pl.splits > 1) {
         const long long tasks = static_cast<long long>(a.R) * a.N * a.Hq;
-        combine_kernel<<<static_cast<unsigned>((tasks + 3) / 4), 128, 0, st>>>(p);
-        e = cudaGetLastError();
+        e = launch_pdl(combine_kernel, dim3(static_cast<unsigned>((tasks + 3) / 4)), dim3(128), 0, st, p);
         if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: combine: %s", cudaGetErrorString(e));
     }
     return DDTREE_OK;

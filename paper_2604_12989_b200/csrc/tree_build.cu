@@ -129,6 +129,7 @@ tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restric
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = B + 1, W = (N + 31) / 32;
 
+    pdl_wait();
     BTRACE(0);
     // ---- 1. merge chunk partials: one warp per draft position ---------------------------------
     for (int i = warp; i < L; i += kWarps) {
@@ -402,16 +403,14 @@ cudaError_t launch_tree_build(int R, int L, int V, int K, int B, const BuildPart
     const float* tmax = reinterpret_cast<const float*>(w + lay.off_tmax);
     const float* wmax = reinterpret_cast<const float*>(w + lay.off_wmax);
     if (dt == DDTREE_F32)
-        tree_build_kernel<float><<<R, kThreads, 0, st>>>(
+        return launch_pdl(tree_build_kernel<float>, dim3(R), dim3(kThreads), 0, st,
             L, V, K, B, lay.chunks, pm, ps, tmax, wmax, static_cast<const float*>(logits), row_stride, root_token, prefix_len,
             n_rows, node_token, node_parent, node_depth, position_ids, anc_mask, first_child, child_count, node_logprob,
             topk_token, topk_logprob);
-    else
-        tree_build_kernel<__nv_bfloat16><<<R, kThreads, 0, st>>>(
+    return launch_pdl(tree_build_kernel<__nv_bfloat16>, dim3(R), dim3(kThreads), 0, st,
             L, V, K, B, lay.chunks, pm, ps, tmax, wmax, static_cast<const __nv_bfloat16*>(logits), row_stride, root_token,
             prefix_len, n_rows, node_token, node_parent, node_depth, position_ids, anc_mask, first_child, child_count,
             node_logprob, topk_token, topk_logprob);
-    return cudaGetLastError();
 }
 
 }  // namespace ddtree
