@@ -182,3 +182,61 @@ def test_bf16_first_call_of_a_fresh_process():
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     res = subprocess.run([sys.executable, "-c", code], cwd=root, capture_output=True, text=True, timeout=600)
     assert res.returncode == 0 and "fresh-process ok" in res.stdout, res.stdout + res.stderr
+
+
+def test_bf16_largest_tree_and_custom_scale():
+    """B = 1024 (1025 rows, 33 mask words, nine 128-key tree tiles), empty prefix, 16 query heads per KV
+    head, a caller-chosen softmax scale and no lse output."""
+    import paper_2604_12989_b200 as dd
+    w = wl.small_workload(R=1, L=12, V=3000, K=6, B=1024, Hq=16, Hkv=1, d=128, dtype="bf16", prefix_lens=(0,), index=41)
+    att, trees = make_case(w)
+    assert trees[0].n_rows == 1025
+    mask = torch.from_numpy(trees[0].mask[None].view(np.int32)).cuda()
+    n_rows = torch.tensor([1025], dtype=torch.int32).cuda()
+    cu = torch.from_numpy(att.cu_prefix).cuda()
+    q, kc, vc, kt, vt = (cases.to_torch(getattr(att, n), True) for n in ("q", "k_cache", "v_cache", "k_tree", "v_tree"))
+    kc = torch.zeros(1, 1, 128, dtype=torch.bfloat16, device="cuda")  # empty prefix: never read
+    vc = torch.zeros_like(kc)
+    out = dd.ddtree_tree_attention(q, kc, vc, [0, 0], cu, kt, vt, mask, n_rows, softmax_scale=0.05)
+    torch.cuda.synchronize()
+    dd.device_status()
+    got = out.float().cpu().numpy().astype(np.float64)
+    rng = np.random.default_rng(0)
+    empty = np.zeros((0, 1, 128))
+    for _ in range(40):
+        i, h = int(rng.integers(0, 1025)), int(rng.integers(0, 16))
+        ref, _ = orc.tree_attention(att.as_f64("q")[0], empty, empty, att.as_f64("k_tree")[0], att.as_f64("v_tree")[0],
+                                    trees[0].mask, 1025, scale=0.05, rows=[i], heads=[h])
+        err = np.abs(got[0, i, h] - ref[0, 0]) / (1 + np.abs(ref[0, 0]))
+        assert err.max() <= 1e-2, (i, h, err.max())
+
+
+def test_bf16_batch_with_an_empty_prefix_and_a_root_only_tree():
+    """Request 0 has no cached context, request 2's tree is the root alone (n_rows = 1)."""
+    w = wl.small_workload(R=3, L=6, V=900, K=3, B=37, Hq=8, Hkv=2, d=128, dtype="bf16", prefix_lens=(0, 700, 130), index=42)
+    att, trees = make_case(w)
+    root_only = orc.compile_tree([], np.zeros((6, 3), np.int64), 5, 130, w.B)
+    assert root_only.n_rows == 1
+    trees[2] = root_only
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse)
+    assert (out[2, 1:] == 0).all()
+
+
+def test_bf16_workspace_too_small_is_refused():
+    import paper_2604_12989_b200 as dd
+    w, att, trees = bf16_case(1, 64, 8, 2, (2000,))
+    mask = torch.from_numpy(np.stack([t.mask for t in trees]).view(np.int32)).cuda()
+    n_rows = torch.tensor([t.n_rows for t in trees], dtype=torch.int32).cuda()
+    q, kc, vc, kt, vt = (cases.to_torch(getattr(att, n), True) for n in ("q", "k_cache", "v_cache", "k_tree", "v_tree"))
+    need = dd.tree_attention_workspace_bytes(1, 64, 8, 2, 128, 1, att.cu_prefix.tolist())
+    assert need > 4096
+    with pytest.raises(dd.DDTreeError) as e:
+        dd.ddtree_tree_attention(q, kc, vc, att.cu_prefix.tolist(), torch.from_numpy(att.cu_prefix).cuda(), kt, vt, mask,
+                                 n_rows, workspace=torch.zeros(4096, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 3
+    with pytest.raises(dd.DDTreeError) as e:  # head_dim 64 has no bf16 kernel
+        dd.ddtree_tree_attention(q[..., :64].contiguous(), kc[..., :64].contiguous(), vc[..., :64].contiguous(),
+                                 att.cu_prefix.tolist(), torch.from_numpy(att.cu_prefix).cuda(),
+                                 kt[..., :64].contiguous(), vt[..., :64].contiguous(), mask, n_rows)
+    assert e.value.status == 2

@@ -208,3 +208,57 @@ def test_argument_errors_launch_nothing():
     with pytest.raises(dd.DDTreeError):
         dd.ddtree_build(x[:, :, 1:], 4, 4, z, z)  # rows not 16-byte aligned
     dd.device_status()
+
+
+def test_build_full_vocab_bf16_logits_ragged_batch():
+    """Drafter logits given as bf16 at full vocabulary size.  The retained logits of every position
+    are placed on the bf16 lattice with irregular gaps (multiples of 0.25 below 64), so the input is
+    exactly representable and the top-B set is still unambiguous."""
+    w = wl.small_workload(R=3, L=16, V=151936, K=8, B=48, prefix_lens=(10, 20, 30), noise=3.0, boost0=8.0,
+                          boost_slope=0.4, index=24)
+    roots = wl.root_tokens(w)
+    for attempt in range(20):
+        rng = np.random.default_rng([24, attempt])
+        xb = wl.round_through_bf16(np.stack([wl.drafter_logits(w, r, "lit", attempt) for r in range(3)]))
+        for r in range(3):
+            for i in range(w.L):
+                top = np.argsort(-xb[r, i], kind="stable")[: w.K + 1]
+                steps = rng.integers(1, 6, w.K + 1) * 0.25
+                vals = 20.0 + np.cumsum(steps[::-1])[::-1]  # strictly decreasing, all multiples of 0.25 in (20, 30)
+                xb[r, i, top] = vals.astype(np.float32)
+        assert np.array_equal(wl.round_through_bf16(xb), xb)
+        ok = all(orc.boundary_gap(orc.top_k(xb[r], w.K)[1], w.B) >= 1e-3 for r in range(3))
+        if ok:
+            break
+    else:
+        pytest.skip("no draw with an unambiguous top-B set")
+    trees = cases.oracle_trees(w, xb, roots)
+    tree = run_build(w, xb, roots, bf16_logits=True)
+    for r in range(3):
+        cases.tree_arrays_equal(trees[r], tree, r)
+        assert trees[r].depth.max() >= 2
+
+
+def test_accept_ragged_vocab_tail_bf16():
+    """V = 5003 in bf16: rows are padded to 16-byte starts, the last 3 elements are read one by one."""
+    import paper_2604_12989_b200 as dd
+    w = wl.small_workload(R=2, L=5, V=5003, K=3, B=25, prefix_lens=(1, 2), dtype="bf16", index=25)
+    logits = np.stack([wl.drafter_logits(w, r, "peak") for r in range(2)])
+    roots = wl.root_tokens(w)
+    trees = cases.oracle_trees(w, logits, roots)
+    tree = run_build(w, logits, roots)
+    tl = np.stack([wl.target_logits(w, trees[r].depth, r, "peak") for r in range(2)])
+    for r in range(2):  # put the maximum of some rows into the ragged tail
+        tl[r, 0, 5002] = wl.f32_to_bf16_bits(np.array([80.0], np.float32))[0]
+        tl[r, 1, 5000] = wl.f32_to_bf16_bits(np.array([90.0], np.float32))[0]
+    t = cases.to_torch(tl, True)
+    t = torch.nn.functional.pad(t, (0, 5))[:, :, :5003]
+    acc = dd.ddtree_accept(t, w.L, tree.node_token, tree.node_parent, tree.n_rows)
+    torch.cuda.synchronize()
+    for r in range(2):
+        choice = orc.node_argmax(wl.bf16_to_f64(tl[r]))
+        assert choice[0] == 5002 and choice[1] == 5000
+        n = trees[r].n_rows
+        np.testing.assert_array_equal(acc.node_argmax[r].cpu().numpy()[:n], choice[:n])
+        want = orc.accept_walk(trees[r].token, trees[r].parent, n, choice)
+        assert int(acc.accept_len[r]) == want.accept_len and int(acc.bonus_token[r]) == want.bonus_token
