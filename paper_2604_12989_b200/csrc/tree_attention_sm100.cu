@@ -68,8 +68,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Non-blocking test of a phase.  try_wait may park the thread for a while and costs a couple of
+// hundred cycles even when the phase has long completed; test_wait answers at once, so every wait
+// starts with it and several barriers can be tested back to back.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait.  Returns false when it gave up (or another thread of the CTA already did).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    if (mbar_test(bar, parity)) return true;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 32) {
@@ -201,7 +214,19 @@ __device__ __forceinline__ void trace_clk(int idx) {
     }
 }
 #define TRACE_CLK(idx) trace_clk(idx)
+// Low-overhead time stamps: clock64 into registers for two steady-state tiles, written out once
+// after the loop (a stamp that writes to global memory costs ~300 cycles and distorts the loop).
+constexpr int kStampTile = 8;
+#define STAMP_DECL long long stamp_[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
+#define STAMP(cond, i) do { if (cond) { long long t_; asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_)); stamp_[i] = t_; } } while (0)
+#define STAMP_FLUSH(cond, base) do { if ((cond) && g_trace) { \
+        const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); \
+        for (int i_ = 0; i_ < 16; ++i_) g_trace[cta_ * 64 + (base) + i_] = static_cast<unsigned long long>(stamp_[i_]); } } while (0)
 #else
+constexpr int kStampTile = 8;
+#define STAMP_DECL ((void)0)
+#define STAMP(cond, i) ((void)0)
+#define STAMP_FLUSH(cond, base) ((void)0)
 #define TRACE(idx) ((void)0)
 #define TRACE_CLK(idx) ((void)0)
 #endif
@@ -230,6 +255,11 @@ struct KernelParams {
     float scale_log2;
 };
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -242,6 +272,20 @@ __device__ __forceinline__ float ex2(float x) {
 // the exponentials already saturate.
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return __byte_perm(__float_as_uint(a) + 0x8000u, __float_as_uint(b) + 0x8000u, 0x7632);
+}
+
+// Exponentials of score columns [kBegin, kEnd) of one thread relative to the reference m_use, packed to
+// bf16 pairs (low half = even key), and their sum added to rowsum.
+template <int kBegin, int kEnd>
+__device__ __forceinline__ void exp_block(const uint32_t (&sv)[64], uint32_t (&pk)[32], float& rowsum, float scale_log2,
+                                          float m_use) {
+#pragma unroll
+    for (int c = kBegin; c < kEnd; c += 2) {
+        const float e0 = ex2(fmaf(__uint_as_float(sv[c]), scale_log2, -m_use));
+        const float e1 = ex2(fmaf(__uint_as_float(sv[c + 1]), scale_log2, -m_use));
+        rowsum += e0 + e1;
+        pk[c >> 1] = pack_bf16(e0, e1);
+    }
 }
 
 // Replace the scores of invisible keys by -inf: bit c of `word` tells whether key c of this
@@ -401,17 +445,29 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             if (elect_one()) issue_qk(j);
             __syncwarp();
         }
+        STAMP_DECL;
         for (int j = 0; j < my_tiles && ok; ++j) {
+            const bool st8 = j == kStampTile, st9 = j == kStampTile + 1;
+            STAMP(st8 || st9, st8 ? 0 : 3);
             // One burst per tile: O_h += P_h V_h for both column halves of tile j, then the scores of
             // tile j+2 into the S buffer those P halves sat in.  The tensor pipe pays a start-up
             // latency of a few hundred cycles whenever it has drained, so bursts are kept long.
             const int s = j % kStages, b = j % kSBufs;
             const bool more = j + kSBufs < my_tiles;
-            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.v_full[s]), (j / kStages) & 1, abort_flag)) &&
-                 (!more || wait_k(j + kSBufs)) &&
-                 __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[b][0]), (j / kSBufs) & 1, abort_flag)) &&
-                 __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[b][1]), (j / kSBufs) & 1, abort_flag));
-            if (!ok) break;
+            // the four tests are independent instructions: their latencies overlap, and the tensor pipe
+            // drains within ~150 cycles of the last issue, so this check must be short
+            const bool k_ok = !more || mbar_test(smem_u32(&sm.k_full[(j + kSBufs) % kStages]), ((j + kSBufs) / kStages) & 1);
+            const bool ready = mbar_test(smem_u32(&sm.v_full[s]), (j / kStages) & 1) & k_ok &
+                               mbar_test(smem_u32(&sm.p_ready[b][0]), (j / kSBufs) & 1) &
+                               mbar_test(smem_u32(&sm.p_ready[b][1]), (j / kSBufs) & 1);
+            if (!__all_sync(kFull, ready)) {
+                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.v_full[s]), (j / kStages) & 1, abort_flag)) &&
+                     (!more || wait_k(j + kSBufs)) &&
+                     __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[b][0]), (j / kSBufs) & 1, abort_flag)) &&
+                     __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[b][1]), (j / kSBufs) & 1, abort_flag));
+                if (!ok) break;
+            }
+            STAMP(st8 || st9, st8 ? 1 : 4);
             tc_fence_after();
             const uint64_t vd = v_desc0 + static_cast<uint64_t>(s) * (kTileBytes >> 4);
             const uint32_t a_p = tmem + kColS + b * kTile;  // bf16 P: half h in columns [64h, 64h+32)
@@ -434,7 +490,9 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                 if (more) issue_qk(j + kSBufs);
             }
             __syncwarp();
+            STAMP(st8 || st9, st8 ? 2 : 5);
         }
+        STAMP_FLUSH(lane == 0, 0);
     } else {
         // ---- softmax: 256 threads; thread (wt, half) owns key columns [64*half, 64*half+64) of row wt in
         //      every tile, with its own reference maximum, sum and O accumulator: the two halves of a
@@ -449,16 +507,34 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         float m_run = -CUDART_INF_F;   // reference maximum of the exponentials, scaled log2 units
         float l_run = 0.f;
         bool ok = true;
+        bool s_ready = false;    // result of the early test of s_full for the coming tile
+        bool preloaded = false;  // the TMEM load of the coming tile's scores is already in flight
+        uint32_t sv[64];
+        STAMP_DECL;
         for (int j = 0; j < my_tiles && ok; ++j) {
             const int t = t_begin + j, b = j % kSBufs;
             const uint32_t s_addr = lane_addr + kColS + b * kTile + half * 64;
-            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.s_full[b]), (j / kSBufs) & 1, abort_flag));
-            if (!ok) break;  // warp-uniform: the TMEM loads/stores below need the whole warp
+            const bool st8 = j == kStampTile;
+            STAMP(st8, 0);
+            STAMP(j == kStampTile + 1, 8);
+            STAMP(j == kStampTile + 2, 9);
+            // Barrier tests, votes and TMEM round trips cost 150-300 cycles each, during which the two
+            // softmax warps of an SM sub-partition (always in the same phase) leave it idle.  So they are
+            // taken off the critical path: the barriers of the coming tile are tested in the middle of
+            // this tile's exponentials, and its scores are requested from TMEM before this tile's P is
+            // stored; the top of the loop normally finds the load in flight.
+            if (!preloaded) {
+                if (!__all_sync(kFull, s_ready)) {
+                    ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.s_full[b]), (j / kSBufs) & 1, abort_flag));
+                    if (!ok) break;  // warp-uniform: the TMEM loads/stores below need the whole warp
+                }
+                tc_fence_after();
+                TMEM_LD32(sv, 0, s_addr);
+                TMEM_LD32(sv, 32, s_addr + 32);
+            }
             if (wt == 0 && j < 5) TRACE(half ? 20 + 2 * j : 4 + 3 * j);
-            tc_fence_after();
-            uint32_t sv[64];
-            TMEM_LD32(sv, 0, s_addr);
-            TMEM_LD32(sv, 32, s_addr + 32);
+            STAMP(st8, 1);
+            bool saw_o_done = j == 0;  // phase j-1 of o_done must be observed exactly once per tile (see below)
 
             // visibility of this thread's 64 keys
             uint32_t vis0 = kFull, vis1 = kFull;
@@ -477,22 +553,41 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                 vis1 = w0 + 1 < p.W ? mrow[w0 + 1] : 0u;
             }
             tmem_wait_ld();
+            STAMP(st8, 2);
             if (!all_visible) { mask32(sv, 0, vis0); mask32(sv, 32, vis1); }
-            float mx = -CUDART_INF_F;
+            // Optimistic pass: exponentials relative to the reference maximum as it stands.  P keeps its
+            // relative precision whatever the reference (bf16 has the exponent range of fp32), so the
+            // reference only has to keep the sums away from overflow: it is revisited when a row sum
+            // exceeds 2^24 (or is not finite), and on the first tile, where there is none yet.
+            float rowsum = 0.f;
+            uint32_t pk[32];
+            {
+                const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
+                exp_block<0, 32>(sv, pk, rowsum, p.scale_log2, m_use);
+                // early tests of the coming tile's barriers (results are consumed further down)
+                s_ready = j + 1 < my_tiles && mbar_test(smem_u32(&sm.s_full[(j + 1) % kSBufs]), ((j + 1) / kSBufs) & 1);
+                if (!saw_o_done) saw_o_done = mbar_test(smem_u32(&sm.o_done[half]), (j - 1) & 1);
+                exp_block<32, 64>(sv, pk, rowsum, p.scale_log2, m_use);
+            }
+            STAMP(st8, 3);
+            const bool revisit = m_run == -CUDART_INF_F || !(rowsum < 16777216.f);
+            if (__any_sync(kFull, revisit)) {
+                // exact maximum of my 64 scores; the reference moves only when the maximum outgrew it by 2^8
+                float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-            for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
-            if (tid == 0 && j < 5) TRACE(5 + 3 * j);
-            // move the reference maximum only when the maximum outgrew it by 2^8: the exponentials
-            // then stay below 2^8 and the O accumulator rarely needs rescaling
-            const float m_tile = mx * p.scale_log2;
-            const bool bump = m_tile > m_run + 8.f;
-            bool saw_o_done = j == 0;  // phase j-1 of o_done must be observed exactly once per tile (see below)
-            if (__any_sync(kFull, bump)) {
+                for (int c = 0; c < 64; c += 8)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mx4[k] = max3(mx4[k], __uint_as_float(sv[c + 2 * k]), __uint_as_float(sv[c + 2 * k + 1]));
+                const float m_tile = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * p.scale_log2;
+                const bool bump = m_tile > m_run + 8.f;
                 const float alpha = bump ? ex2(m_run - m_tile) : 1.f;
                 if (bump) { l_run *= alpha; m_run = m_tile; }
-                if (j > 0) {  // O_half holds the sum over the earlier tiles: wait for it, rescale my row
-                    ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[half]), (j - 1) & 1, abort_flag));
-                    if (!ok) break;
+                if (j > 0 && __any_sync(kFull, bump)) {  // O_half holds the sum over the earlier tiles: rescale my row
+                    if (!__all_sync(kFull, saw_o_done)) {
+                        ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[half]), (j - 1) & 1, abort_flag));
+                        if (!ok) break;
+                    }
                     saw_o_done = true;
                     tc_fence_after();
 #pragma unroll
@@ -505,34 +600,39 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                         TMEM_ST32(o_addr + c0, ov, 0);
                     }
                 }
+                const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
+                rowsum = 0.f;
+                exp_block<0, 64>(sv, pk, rowsum, p.scale_log2, m_use);
             }
-            const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
-
-            // exponentials, row sum, bf16 P written over the first 32 of my 64 score columns
-            float rowsum = 0.f;
-            uint32_t pk[32];
-#pragma unroll
-            for (int c = 0; c < 64; c += 2) {
-                const float e0 = ex2(fmaf(__uint_as_float(sv[c]), p.scale_log2, -m_use));
-                const float e1 = ex2(fmaf(__uint_as_float(sv[c + 1]), p.scale_log2, -m_use));
-                rowsum += e0 + e1;
-                pk[c >> 1] = pack_bf16(e0, e1);  // low half = even key
+            STAMP(st8, 4);
+            // the scores are consumed: request the coming tile's (other S buffer) before storing P
+            preloaded = __all_sync(kFull, s_ready);
+            if (preloaded) {
+                tc_fence_after();
+                const uint32_t s_next = lane_addr + kColS + ((j + 1) % kSBufs) * kTile + half * 64;
+                TMEM_LD32(sv, 0, s_next);
+                TMEM_LD32(sv, 32, s_next + 32);
             }
             TMEM_ST32(s_addr, pk, 0);
             l_run += rowsum;
             tmem_wait_st();
+            STAMP(st8, 5);
             // A parity wait cannot tell phase j-1 from phase j-3: a thread that skipped phases could
             // sail through a later wait while the product it needs is still running.  So every tile
             // observes the previous tile's o_done, here at the latest (by now it has long completed).
-            if (!saw_o_done) {
+            if (!__all_sync(kFull, saw_o_done)) {
                 ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[half]), (j - 1) & 1, abort_flag));
                 if (!ok) break;
             }
+            STAMP(st8, 6);
             tc_fence_before();
             mbar_arrive(smem_u32(&sm.p_ready[b][half]));
+            STAMP(st8, 7);
             if (wt == 0 && j < 5) TRACE(half ? 21 + 2 * j : 6 + 3 * j);
         }
 
+        if (preloaded) tmem_wait_ld();  // only when the loop was left early: no load may outlive the TMEM allocation
+        STAMP_FLUSH(wt == 0, half ? 32 : 16);
         // ---- epilogue: merge the two halves, O -> shared memory (swizzled rows) -> coalesced stores --
         for (int h = 0; h < 2 && ok; ++h)
             ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[h]), (my_tiles - 1) & 1, abort_flag));
