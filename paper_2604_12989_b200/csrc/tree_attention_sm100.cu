@@ -16,11 +16,12 @@
 //              score buffers; O_h += P_h V_h (P read from TMEM, V as an MN-major shared-memory
 //              operand) as soon as half h of the tile is ready; owns the TMEM allocation
 // The ancestor bitmask is applied only on tree tiles; prefix tiles need at most a length test on
-// the request's last tile.  Each split writes un-normalised fp32 partials; a combine kernel merges
-// them by log-sum-exp.  Every wait is bounded: when one gives up, the CTA raises a flag in the
+// the request's last tile.  Each split writes its normalised rows (fp16) with their reference maximum
+// and sum; a combine kernel merges them by log-sum-exp.  Every wait is bounded: when one gives up, the CTA raises a flag in the
 // device status word, drains its copies and leaves without touching its outputs.
 #include "common.cuh"
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <math_constants.h>
 #include <mutex>
 #include <unordered_map>
@@ -221,7 +222,7 @@ constexpr int kStampTile = 8;
 #define STAMP(cond, i) do { if (cond) { long long t_; asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_)); stamp_[i] = t_; } } while (0)
 #define STAMP_FLUSH(cond, base) do { if ((cond) && g_trace) { \
         const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); \
-        for (int i_ = 0; i_ < 16; ++i_) g_trace[cta_ * 64 + (base) + i_] = static_cast<unsigned long long>(stamp_[i_]); } } while (0)
+        for (int i_ = 0; i_ < 16; ++i_) if (stamp_[i_]) g_trace[cta_ * 64 + (base) + i_] = static_cast<unsigned long long>(stamp_[i_]); } } while (0)
 #else
 constexpr int kStampTile = 8;
 #define STAMP_DECL ((void)0)
@@ -248,7 +249,7 @@ struct KernelParams {
     const int32_t* n_rows;
     __nv_bfloat16* out;
     float* lse;
-    float* part_o;   // [S, R, Hkv, rows_pad, 128]
+    __half* part_o;  // [S, R, Hkv, rows_pad, 128]: each split's O divided by its own sum, fp16
     float2* part_ml; // [S, R, Hkv, rows_pad] (reference max in log2 units, sum)
     uint32_t* status;
     int R, N, W, Hq, Hkv, G, splits, rows_pad;
@@ -653,7 +654,7 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             const float a_self = m_run == -CUDART_INF_F ? 0.f : ex2(m_run - m_row);
             const float a_other = m_o == -CUDART_INF_F ? 0.f : ex2(m_o - m_row);
             l_row = l_run * a_self + l_o * a_other;
-            const float f = direct ? (l_row > 0.f ? 1.f / l_row : 0.f) : 1.f;
+            const float f = l_row > 0.f ? 1.f / l_row : 0.f;  // rows leave normalised, also as split partials
             const float f0 = (half == 0 ? a_self : a_other) * f, f1 = (half == 0 ? a_other : a_self) * f;
             // this thread merges head-dim columns [64*half, 64*half+64) of its row from both accumulators
 #pragma unroll
@@ -680,27 +681,66 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         if (ok) {
             const int rows_valid = min(kTile, n * p.G - rt * kTile);
             if (direct) {
-                // 16 chunks of 8 bf16 per row
-                for (int idx = tid; idx < rows_valid * 16; idx += kSoftmaxThreads) {
-                    const int row = idx >> 4, c8 = idx & 15;
-                    const float4 a = stage[row * 32 + ((2 * c8) ^ (row & 31))];
-                    const float4 bq = stage[row * 32 + ((2 * c8 + 1) ^ (row & 31))];
-                    const __nv_bfloat162 b0 = __floats2bfloat162_rn(a.x, a.y), b1 = __floats2bfloat162_rn(a.z, a.w);
-                    const __nv_bfloat162 b2 = __floats2bfloat162_rn(bq.x, bq.y), b3 = __floats2bfloat162_rn(bq.z, bq.w);
-                    const int gr = rt * kTile + row;
-                    const size_t orow = ((static_cast<size_t>(r) * p.N + gr / p.G) * p.Hq + kvh * p.G + gr % p.G) * kTile;
-                    *reinterpret_cast<uint4*>(p.out + orow + c8 * 8) =
-                        make_uint4(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1),
-                                   *reinterpret_cast<const uint32_t*>(&b2), *reinterpret_cast<const uint32_t*>(&b3));
+                // 16 chunks of 8 bf16 per row; four chunks per thread and step so that the shared-memory
+                // loads of a step are in flight together
+                const int total = rows_valid * 16;
+                for (int base = tid; base < total; base += kSoftmaxThreads * 4) {
+                    float4 a[4], bq[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int idx = base + u * kSoftmaxThreads;
+                        if (idx < total) {
+                            const int row = idx >> 4, c8 = idx & 15;
+                            a[u] = stage[row * 32 + ((2 * c8) ^ (row & 31))];
+                            bq[u] = stage[row * 32 + ((2 * c8 + 1) ^ (row & 31))];
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int idx = base + u * kSoftmaxThreads;
+                        if (idx < total) {
+                            const int row = idx >> 4, c8 = idx & 15;
+                            const __nv_bfloat162 b0 = __floats2bfloat162_rn(a[u].x, a[u].y), b1 = __floats2bfloat162_rn(a[u].z, a[u].w);
+                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(bq[u].x, bq[u].y), b3 = __floats2bfloat162_rn(bq[u].z, bq[u].w);
+                            const int gr = rt * kTile + row;
+                            const size_t orow = ((static_cast<size_t>(r) * p.N + gr / p.G) * p.Hq + kvh * p.G + gr % p.G) * kTile;
+                            *reinterpret_cast<uint4*>(p.out + orow + c8 * 8) =
+                                make_uint4(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1),
+                                           *reinterpret_cast<const uint32_t*>(&b2), *reinterpret_cast<const uint32_t*>(&b3));
+                        }
+                    }
                 }
                 if (half == 0 && valid && p.lse)
                     p.lse[(static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + grow % p.G] =
                         (m_row + log2f(l_row)) / kLog2e;
             } else {
-                float4* dst = reinterpret_cast<float4*>(p.part_o + part_row0 * kTile);
-                for (int idx = tid; idx < rows_valid * 32; idx += kSoftmaxThreads) {
-                    const int row = idx >> 5, g4 = idx & 31;
-                    dst[idx] = stage[row * 32 + (g4 ^ (row & 31))];
+                // Split partial: the normalised row in fp16 (values are averages of V rows, so fp16's
+                // 11 bits are finer than the bf16 rounding of the final output; half the bytes of fp32,
+                // and the L2 write rate is what this step is bound by) plus (reference maximum, sum)
+                __half* dst = p.part_o + part_row0 * kTile;
+                const int total = rows_valid * 16;
+                for (int base = tid; base < total; base += kSoftmaxThreads * 4) {
+                    float4 a[4], bq[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int idx = base + u * kSoftmaxThreads;
+                        if (idx < total) {
+                            const int row = idx >> 4, c8 = idx & 15;
+                            a[u] = stage[row * 32 + ((2 * c8) ^ (row & 31))];
+                            bq[u] = stage[row * 32 + ((2 * c8 + 1) ^ (row & 31))];
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int idx = base + u * kSoftmaxThreads;
+                        if (idx < total) {
+                            const __half2 h0 = __floats2half2_rn(a[u].x, a[u].y), h1 = __floats2half2_rn(a[u].z, a[u].w);
+                            const __half2 h2 = __floats2half2_rn(bq[u].x, bq[u].y), h3 = __floats2half2_rn(bq[u].z, bq[u].w);
+                            *reinterpret_cast<uint4*>(dst + idx * 8) =
+                                make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
+                                           *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
+                        }
+                    }
                 }
                 if (half == 0) p.part_ml[part_row0 + wt] = make_float2(m_row, l_row);
             }
@@ -731,8 +771,8 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     }
 }
 
-// Merge the per-split partials of one (request, row, head): out = sum_s w_s O_s / sum_s w_s l_s
-// with w_s = 2^(m_s - max m).  One warp per output row; lane s first fetches split s's (m, l), so
+// Merge the per-split partials of one (request, row, head): out = sum_s w_s l_s O_s / sum_s w_s l_s
+// with O_s the split's normalised row and w_s = 2^(m_s - max m).  One warp per output row; lane s first fetches split s's (m, l), so
 // all splits' loads are in flight together (at most 32 splits).
 __global__ void __launch_bounds__(128)
 combine_kernel(const KernelParams p) {
@@ -753,18 +793,21 @@ combine_kernel(const KernelParams p) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
     const float w = ml.y > 0.f ? exp2f(ml.x - M) : 0.f;  // an empty split never wrote its O row
-    float l = w * ml.y;
+    const float wl = w * ml.y;
+    float l = wl;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(kFull, l, o);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    const float* po = p.part_o + row0 * kTile + lane * 4;
+    const __half* po = p.part_o + row0 * kTile + lane * 4;
 #pragma unroll 4
     for (int s = 0; s < p.splits; ++s) {
-        const float ws = __shfl_sync(kFull, w, s);
+        const float ws = __shfl_sync(kFull, wl, s);
         if (ws == 0.f) continue;  // warp-uniform
-        const float4 o = *reinterpret_cast<const float4*>(po + s * split_stride * kTile);
-        acc[0] = fmaf(ws, o.x, acc[0]); acc[1] = fmaf(ws, o.y, acc[1]);
-        acc[2] = fmaf(ws, o.z, acc[2]); acc[3] = fmaf(ws, o.w, acc[3]);
+        const uint2 raw = *reinterpret_cast<const uint2*>(po + s * split_stride * kTile);
+        const float2 o01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
+        const float2 o23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+        acc[0] = fmaf(ws, o01.x, acc[0]); acc[1] = fmaf(ws, o01.y, acc[1]);
+        acc[2] = fmaf(ws, o23.x, acc[2]); acc[3] = fmaf(ws, o23.y, acc[3]);
     }
     const float inv = 1.f / l;
     const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv);
@@ -873,7 +916,7 @@ Plan make_plan(const AttnArgs& a) {
     }
     pl.splits = s;
     const size_t rows = static_cast<size_t>(s) * a.R * a.Hkv * pl.rows_pad;
-    pl.off_ml = (rows * kTile * 4 + 255) / 256 * 256;
+    pl.off_ml = (rows * kTile * 2 + 255) / 256 * 256;
     pl.total = pl.off_ml + (rows * 8 + 255) / 256 * 256;
     if (s == 1) { pl.off_ml = 0; pl.total = 256; }
     return pl;
@@ -908,7 +951,7 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t*, void* ws, size
     KernelParams p;
     p.cu_prefix = a.cu_prefix; p.anc_mask = a.anc_mask; p.n_rows = a.n_rows;
     p.out = static_cast<__nv_bfloat16*>(a.out); p.lse = a.lse;
-    p.part_o = reinterpret_cast<float*>(ws);
+    p.part_o = reinterpret_cast<__half*>(ws);
     p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(ws) + pl.off_ml);
     p.status = device_status_word();
     if (!p.status) return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: no device status word");
