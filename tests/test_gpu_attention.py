@@ -115,6 +115,22 @@ def test_bf16_short_prefixes_and_sentinel_values(P):
     compare(w, att, trees, out, lse)
 
 
+@pytest.mark.parametrize("profile", ["growing", "exploding", "shrinking"])
+def test_bf16_scores_that_outgrow_the_reference_maximum(profile):
+    # The kernel exponentiates a tile against the reference maximum it already has and looks at the
+    # exact maximum only when a row sum comes near overflow.  Keys whose scale changes from one
+    # 128-key tile to the next force that path: "growing" lifts the scores by ~2^30 per tile (row
+    # sums pass 2^24), "exploding" by more than 2^128 (the optimistic exponentials are infinite),
+    # "shrinking" puts the largest scores first (reference far above everything that follows).
+    w, att, trees = bf16_case(1, 40, 8, 2, (6 * 128 + 17,), seed=11)
+    k = wl.bf16_to_f64(att.k_cache).astype(np.float32)
+    tiles = np.arange(k.shape[0]) // 128
+    factor = {"growing": 1.0 + 6.0 * tiles, "exploding": 1.0 + 40.0 * tiles, "shrinking": 40.0 / (1.0 + 6.0 * tiles)}[profile]
+    att.k_cache = wl.f32_to_bf16_bits(k * factor[:, None, None].astype(np.float32))
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse)
+
+
 @pytest.mark.parametrize("G,Hkv", [(1, 2), (2, 2), (4, 1), (8, 1), (16, 1)])
 def test_bf16_group_sizes(G, Hkv):
     w, att, trees = bf16_case(1, 40, G * Hkv, Hkv, (200,), seed=G)
