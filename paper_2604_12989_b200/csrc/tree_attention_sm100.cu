@@ -234,10 +234,10 @@ constexpr int kStampTile = 8;
 
 struct Smem {
     uint8_t q[kTileBytes];
-    uint8_t k[kStages][kTileBytes];   // after the last MMA, k[0..1] double as the 64 KB output staging buffer
+    uint8_t k[kStages][kTileBytes];
     uint8_t v[kStages][kTileBytes];
     uint64_t q_full, k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
-    uint64_t s_full[kSBufs], p_ready[kSBufs][2], o_done[2], fin[2];
+    uint64_t s_full[kSBufs], p_ready[kSBufs][2], o_done[2], fin;
     float xm[2][kTile], xl[2][kTile]; // [column half][row]: reference maximum and sum, exchanged at the end
     uint32_t tmem_base;
     uint32_t abort;
@@ -367,10 +367,8 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             mbar_init(smem_u32(&sm.p_ready[b][0]), kGroupThreads);
             mbar_init(smem_u32(&sm.p_ready[b][1]), kGroupThreads);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&sm.o_done[b]), 1);
-            mbar_init(smem_u32(&sm.fin[b]), kSoftmaxThreads);
-        }
+        for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&sm.o_done[b]), 1);
+        mbar_init(smem_u32(&sm.fin), kSoftmaxThreads);
         sm.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -633,20 +631,21 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         }
 
         if (preloaded) tmem_wait_ld();  // only when the loop was left early: no load may outlive the TMEM allocation
-        STAMP_FLUSH(wt == 0, half ? 32 : 16);
-        // ---- epilogue: merge the two halves, O -> shared memory (swizzled rows) -> coalesced stores --
+        STAMP(true, 10);
+        // ---- epilogue: merge the two halves and write each row's 16-bit values straight from registers ----
         for (int h = 0; h < 2 && ok; ++h)
             ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[h]), (my_tiles - 1) & 1, abort_flag));
         if (tid == 0) TRACE(46);
-        float4* stage = reinterpret_cast<float4*>(sm.k[0]);  // [128 rows][32 float4], free once all MMAs are done
+        STAMP(true, 11);
         const bool direct = p.splits == 1;
         if (ok) {
             tc_fence_after();
             sm.xm[half][wt] = m_run;
             sm.xl[half][wt] = l_run;
-            mbar_arrive(smem_u32(&sm.fin[0]));
-            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.fin[0]), 0, abort_flag));
+            mbar_arrive(smem_u32(&sm.fin));
+            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.fin), 0, abort_flag));
         }
+        STAMP(true, 12);
         float l_row = 0.f, m_row = -CUDART_INF_F;
         if (ok) {
             const float m_o = sm.xm[half ^ 1][wt], l_o = sm.xl[half ^ 1][wt];
@@ -656,95 +655,55 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             l_row = l_run * a_self + l_o * a_other;
             const float f = l_row > 0.f ? 1.f / l_row : 0.f;  // rows leave normalised, also as split partials
             const float f0 = (half == 0 ? a_self : a_other) * f, f1 = (half == 0 ? a_other : a_self) * f;
-            // this thread merges head-dim columns [64*half, 64*half+64) of its row from both accumulators
+            // this thread merges head-dim columns [64*half, 64*half+64) of its row from both accumulators,
+            // rounds them to 16 bits and writes its 128 contiguous bytes itself: to the output (bf16)
+            // when this CTA saw the whole KV range, else to the split partials (fp16: the rows are
+            // averages of V rows, so fp16's 11 bits are finer than the bf16 rounding of the final output).
+            // (An SM stores ~32 bytes per clock whatever the route: staging the rows for coalesced stores
+            // or for one bulk tensor store was measured and takes the same time.)
+            uint16_t* dst16;
+            if (direct) {
+                dst16 = reinterpret_cast<uint16_t*>(p.out) +
+                        ((static_cast<size_t>(r) * p.N + (valid ? node : 0)) * p.Hq + kvh * p.G + grow % p.G) * kTile + half * 64;
+            } else {
+                dst16 = reinterpret_cast<uint16_t*>(p.part_o) + (part_row0 + wt) * kTile + half * 64;
+            }
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t o0[32], o1[32];
+                uint32_t o0[32], o1[32], w16[16];
                 TMEM_LD32(o0, 0, lane_addr + kColO + half * 64 + c0);
                 TMEM_LD32(o1, 0, lane_addr + kColO + kTile + half * 64 + c0);
                 tmem_wait_ld();
+                STAMP(c0 == 0, 13);
 #pragma unroll
-                for (int q4 = 0; q4 < 8; ++q4) {
-                    const int g4 = (half * 64 + c0) / 4 + q4;  // float4 group within the row
-                    float4 vv;
-                    vv.x = fmaf(__uint_as_float(o1[q4 * 4]), f1, __uint_as_float(o0[q4 * 4]) * f0);
-                    vv.y = fmaf(__uint_as_float(o1[q4 * 4 + 1]), f1, __uint_as_float(o0[q4 * 4 + 1]) * f0);
-                    vv.z = fmaf(__uint_as_float(o1[q4 * 4 + 2]), f1, __uint_as_float(o0[q4 * 4 + 2]) * f0);
-                    vv.w = fmaf(__uint_as_float(o1[q4 * 4 + 3]), f1, __uint_as_float(o0[q4 * 4 + 3]) * f0);
-                    stage[wt * 32 + (g4 ^ (wt & 31))] = vv;
+                for (int q = 0; q < 16; ++q) {
+                    const float a = fmaf(__uint_as_float(o1[2 * q]), f1, __uint_as_float(o0[2 * q]) * f0);
+                    const float b = fmaf(__uint_as_float(o1[2 * q + 1]), f1, __uint_as_float(o0[2 * q + 1]) * f0);
+                    if (direct) {
+                        const __nv_bfloat162 t2 = __floats2bfloat162_rn(a, b);
+                        w16[q] = *reinterpret_cast<const uint32_t*>(&t2);
+                    } else {
+                        const __half2 t2 = __floats2half2_rn(a, b);
+                        w16[q] = *reinterpret_cast<const uint32_t*>(&t2);
+                    }
+                }
+                if (valid) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        *reinterpret_cast<uint4*>(dst16 + c0 + 8 * u) = make_uint4(w16[4 * u], w16[4 * u + 1], w16[4 * u + 2], w16[4 * u + 3]);
                 }
             }
-            mbar_arrive(smem_u32(&sm.fin[1]));
-            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.fin[1]), 0, abort_flag));
+            if (half == 0 && valid) {
+                if (direct) {
+                    if (p.lse) p.lse[(static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + grow % p.G] = (m_row + log2f(l_row)) / kLog2e;
+                } else {
+                    p.part_ml[part_row0 + wt] = make_float2(m_row, l_row);
+                }
+            }
         }
+        STAMP(true, 14);
+        STAMP_FLUSH(wt == 0, half ? 32 : 16);
         if (tid == 0) TRACE(47);
-        if (ok) {
-            const int rows_valid = min(kTile, n * p.G - rt * kTile);
-            if (direct) {
-                // 16 chunks of 8 bf16 per row; four chunks per thread and step so that the shared-memory
-                // loads of a step are in flight together
-                const int total = rows_valid * 16;
-                for (int base = tid; base < total; base += kSoftmaxThreads * 4) {
-                    float4 a[4], bq[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int idx = base + u * kSoftmaxThreads;
-                        if (idx < total) {
-                            const int row = idx >> 4, c8 = idx & 15;
-                            a[u] = stage[row * 32 + ((2 * c8) ^ (row & 31))];
-                            bq[u] = stage[row * 32 + ((2 * c8 + 1) ^ (row & 31))];
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int idx = base + u * kSoftmaxThreads;
-                        if (idx < total) {
-                            const int row = idx >> 4, c8 = idx & 15;
-                            const __nv_bfloat162 b0 = __floats2bfloat162_rn(a[u].x, a[u].y), b1 = __floats2bfloat162_rn(a[u].z, a[u].w);
-                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(bq[u].x, bq[u].y), b3 = __floats2bfloat162_rn(bq[u].z, bq[u].w);
-                            const int gr = rt * kTile + row;
-                            const size_t orow = ((static_cast<size_t>(r) * p.N + gr / p.G) * p.Hq + kvh * p.G + gr % p.G) * kTile;
-                            *reinterpret_cast<uint4*>(p.out + orow + c8 * 8) =
-                                make_uint4(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1),
-                                           *reinterpret_cast<const uint32_t*>(&b2), *reinterpret_cast<const uint32_t*>(&b3));
-                        }
-                    }
-                }
-                if (half == 0 && valid && p.lse)
-                    p.lse[(static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + grow % p.G] =
-                        (m_row + log2f(l_row)) / kLog2e;
-            } else {
-                // Split partial: the normalised row in fp16 (values are averages of V rows, so fp16's
-                // 11 bits are finer than the bf16 rounding of the final output; half the bytes of fp32,
-                // and the L2 write rate is what this step is bound by) plus (reference maximum, sum)
-                __half* dst = p.part_o + part_row0 * kTile;
-                const int total = rows_valid * 16;
-                for (int base = tid; base < total; base += kSoftmaxThreads * 4) {
-                    float4 a[4], bq[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int idx = base + u * kSoftmaxThreads;
-                        if (idx < total) {
-                            const int row = idx >> 4, c8 = idx & 15;
-                            a[u] = stage[row * 32 + ((2 * c8) ^ (row & 31))];
-                            bq[u] = stage[row * 32 + ((2 * c8 + 1) ^ (row & 31))];
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int idx = base + u * kSoftmaxThreads;
-                        if (idx < total) {
-                            const __half2 h0 = __floats2half2_rn(a[u].x, a[u].y), h1 = __floats2half2_rn(a[u].z, a[u].w);
-                            const __half2 h2 = __floats2half2_rn(bq[u].x, bq[u].y), h3 = __floats2half2_rn(bq[u].z, bq[u].w);
-                            *reinterpret_cast<uint4*>(dst + idx * 8) =
-                                make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
-                                           *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
-                        }
-                    }
-                }
-                if (half == 0) p.part_ml[part_row0 + wt] = make_float2(m_row, l_row);
-            }
-        }
     }
 
     // ---- teardown -------------------------------------------------------------------------------
