@@ -275,3 +275,17 @@ def accept_walk(token: np.ndarray, parent: np.ndarray, n_rows: int, choice: np.n
         path.append(nxt)
         cur = nxt
     return Acceptance(len(path), path, [int(token[j]) for j in path], int(choice[cur]))
+
+
+def kv_compact(cache: np.ndarray, tree_rows: np.ndarray, prefix_len: int, path: Sequence[int]) -> np.ndarray:
+    """End of a round (Section 4.4: after the walk only the accepted path stays in
+    the cache): the keys (or values) of the root and of the accepted nodes are
+    appended to the cached context in path order, i.e. the root lands at cache
+    position prefix_len and the i-th accepted node at prefix_len + i, which is
+    the position id it was verified at (its depth).  `cache` is [rows, ...] with
+    at least prefix_len + len(path) + 1 rows; returns the updated copy."""
+    out = cache.copy()
+    out[prefix_len] = tree_rows[0]
+    for i, j in enumerate(path):
+        out[prefix_len + 1 + i] = tree_rows[j]
+    return out

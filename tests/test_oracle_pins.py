@@ -473,3 +473,40 @@ def test_walk_stops_at_leaf_of_full_depth():
     choice = np.concatenate([ct.token[1:], [5]]).astype(np.int32)
     acc = orc.accept_walk(ct.token, ct.parent, ct.n_rows, choice)
     assert acc.accept_len == L and acc.nodes == [1, 2, 3, 4] and acc.bonus_token == 5
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_compacted_cache_is_the_context_the_last_accepted_node_saw(seed):
+    """Section 4.4: after the walk only the accepted path stays cached.  Pinned on the attention
+    itself: the last accepted node attended to prefix + root + ancestors + itself, so plain
+    unmasked attention (torch SDPA) of its query over the first P + accept_len + 1 rows of the
+    compacted cache must give its tree-attention output, and every moved row must sit at the
+    position id it was verified at."""
+    rng = np.random.default_rng(100 + seed)
+    L, V, K, B, P, Hq, Hkv, d = 6, 12, 3, 30, 5 + seed, 4, 2, 8
+    ct = orc.build(random_logits(rng, L, V, 1.0), K, B, 0, P)
+    choice = rng.integers(0, V, B + 1).astype(np.int32)
+    for i in range(ct.n_rows):  # make long accepted paths likely
+        if ct.child_count[i] and rng.random() < 0.85:
+            choice[i] = ct.token[ct.first_child[i] + rng.integers(0, ct.child_count[i])]
+    acc = orc.accept_walk(ct.token, ct.parent, ct.n_rows, choice)
+    N = B + 1
+    q = rng.standard_normal((N, Hq, d))
+    cap = P + L + 1
+    kc, vc = rng.standard_normal((cap, Hkv, d)), rng.standard_normal((cap, Hkv, d))
+    kt, vt = rng.standard_normal((N, Hkv, d)), rng.standard_normal((N, Hkv, d))
+    out, _ = orc.tree_attention(q, kc[:P], vc[:P], kt, vt, ct.mask, ct.n_rows)
+    k2 = orc.kv_compact(kc, kt, P, acc.nodes)
+    v2 = orc.kv_compact(vc, vt, P, acc.nodes)
+    np.testing.assert_array_equal(k2[:P], kc[:P])                       # the context is untouched
+    np.testing.assert_array_equal(k2[P + acc.accept_len + 1:], kc[P + acc.accept_len + 1:])
+    last = acc.nodes[-1] if acc.nodes else 0
+    n_ctx = P + acc.accept_len + 1
+    for h in range(Hq):
+        kv = h // (Hq // Hkv)
+        ks = torch.from_numpy(k2[:n_ctx, kv])[None, None]
+        vs = torch.from_numpy(v2[:n_ctx, kv])[None, None]
+        ref = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(q[last, h])[None, None, None], ks, vs)
+        np.testing.assert_allclose(out[last, h], ref[0, 0, 0].numpy(), atol=1e-12)
+    for i, j in enumerate([0] + acc.nodes):
+        assert ct.position_ids[j] == P + i  # cache row P + i holds the token verified at position P + i
