@@ -198,6 +198,31 @@ int ddtree_accept_static_scratch(const void* target_logits, int dt, int64_t row_
                                  int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
                                  int32_t* bonus_token, int32_t* node_argmax, void* cuda_stream);
 
+/* ------------------------------------------------------------------------------------------
+ * ddtree_kv_compact -- Section 4.4, end of a round: after the walk only the accepted path stays
+ * in the KV cache.  For every layer l and request r the rows of the root (tree row 0) and of the
+ * accept_len[r] accepted nodes are copied, in path order, from this round's tree buffers to the
+ * cache rows dst_row[r], dst_row[r] + 1, ..., so that every token sits at the position id it was
+ * verified at (prefix_len + depth).  Nothing else in the cache is touched.  Pure data movement,
+ * all layers in one launch (one more per 64 layers).
+ *
+ *   k_tree, v_tree   HOST arrays of `layers` DEVICE pointers, each [R, B+1, Hkv, d] (dt)
+ *   k_cache, v_cache HOST arrays of `layers` DEVICE pointers, each [rows, Hkv, d] (dt); the caller
+ *                    guarantees rows > dst_row[r] + accept_len[r] for every r (one launch cannot
+ *                    check capacities it is not told)
+ *   dst_row          DEVICE [R] int64: cache row that receives the root of request r; for the packed
+ *                    layout of ddtree_tree_attention this is cu_prefix[r] + prefix_len[r], which
+ *                    needs spare rows behind each request's prefix (trivially so for R = 1)
+ *   accept_len, accept_nodes   DEVICE, as written by ddtree_accept ([R] and [R, L])
+ * Hkv * d * sizeof(dt) must be a multiple of 16 bytes and all buffers 16-byte aligned.  The pointer
+ * arrays are read during the call only.  Errors: as for the other entry points; nothing is
+ * launched when an argument is refused.
+ * ------------------------------------------------------------------------------------------ */
+int ddtree_kv_compact(int R, int B, int L, int Hkv, int d, int dt, int layers,
+                      const void* const* k_tree, const void* const* v_tree,
+                      void* const* k_cache, void* const* v_cache, const int64_t* dst_row,
+                      const int32_t* accept_len, const int32_t* accept_nodes, void* cuda_stream);
+
 /* Device-side status word of the current device: 0, or DDTREE_ERR_DEVICE_TIMEOUT if a bounded
  * wait inside a kernel of this library gave up since the last call.  Synchronises the device,
  * reads and clears the word. */

@@ -22,6 +22,7 @@ EXPORTS = (
     "ddtree_build_workspace_bytes", "ddtree_build",
     "ddtree_tree_attention_workspace_bytes", "ddtree_tree_attention",
     "ddtree_accept_workspace_bytes", "ddtree_accept", "ddtree_accept_static_scratch",
+    "ddtree_kv_compact",
     "ddtree_device_status",
 )
 
@@ -62,6 +63,8 @@ def lib() -> ctypes.CDLL:
         L.ddtree_accept.argtypes = [vp, i32, i64, i32, i32, i32, i32] + [vp] * 8 + [vp, sz, vp]
         L.ddtree_accept_static_scratch.restype = i32
         L.ddtree_accept_static_scratch.argtypes = [vp, i32, i64, i32, i32, i32, i32] + [vp] * 8 + [vp]
+        L.ddtree_kv_compact.restype = i32
+        L.ddtree_kv_compact.argtypes = [i32] * 7 + [vp] * 7 + [vp]
         L.ddtree_device_status.restype = i32
         L.ddtree_device_status.argtypes = []
         _lib = L
@@ -217,6 +220,28 @@ def ddtree_accept_static_scratch(target_logits, L: int, node_token, node_parent,
         out.accept_nodes.data_ptr(), out.accept_tokens.data_ptr(), out.bonus_token.data_ptr(),
         _ptr(out.node_argmax), _stream(stream)))
     return out
+
+
+def ddtree_kv_compact(k_tree, v_tree, k_cache, v_cache, dst_row, accept_len, accept_nodes, stream=None) -> None:
+    """End of a round: copy the root's and the accepted nodes' K/V rows of every layer to cache rows
+    dst_row[r], dst_row[r]+1, ...  k_tree / v_tree: lists (one entry per layer) of [R, B+1, Hkv, d]
+    tensors; k_cache / v_cache: lists of [rows, Hkv, d] tensors, updated in place; dst_row: int64 [R];
+    accept_len, accept_nodes: as returned by ddtree_accept."""
+    import ctypes as c
+    layers = len(k_tree)
+    assert layers >= 1 and len(v_tree) == layers and len(k_cache) == layers and len(v_cache) == layers
+    R, N, Hkv, d = k_tree[0].shape
+    L = accept_nodes.shape[1]
+    for t in list(k_tree) + list(v_tree):
+        assert t.is_cuda and t.is_contiguous() and tuple(t.shape) == (R, N, Hkv, d) and t.dtype == k_tree[0].dtype
+    for t in list(k_cache) + list(v_cache):
+        assert t.is_cuda and t.is_contiguous() and tuple(t.shape[1:]) == (Hkv, d) and t.dtype == k_tree[0].dtype
+    import torch
+    assert dst_row.dtype == torch.int64 and dst_row.is_cuda and dst_row.numel() == R
+    arr = lambda ts: (c.c_void_p * layers)(*[t.data_ptr() for t in ts])
+    _check(lib().ddtree_kv_compact(R, N - 1, L, Hkv, d, _dtype_code(k_tree[0]), layers, arr(k_tree), arr(v_tree),
+                                   arr(k_cache), arr(v_cache), dst_row.data_ptr(), accept_len.data_ptr(),
+                                   accept_nodes.data_ptr(), _stream(stream)))
 
 
 def device_status() -> None:

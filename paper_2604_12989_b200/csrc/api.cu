@@ -130,6 +130,32 @@ int ddtree_accept(const void* target_logits, int dt, int64_t row_stride_elems, i
     return DDTREE_OK;
 }
 
+int ddtree_kv_compact(int R, int B, int L, int Hkv, int d, int dt, int layers, const void* const* k_tree,
+                      const void* const* v_tree, void* const* k_cache, void* const* v_cache, const int64_t* dst_row,
+                      const int32_t* accept_len, const int32_t* accept_nodes, void* cuda_stream) {
+    if (R < 1 || B < 1 || L < 1 || Hkv < 1 || d < 1 || layers < 1)
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_kv_compact: R, B, L, Hkv, d, layers must be >= 1");
+    if (B > kMaxB) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_kv_compact: B %d > %d", B, kMaxB);
+    if (L > kMaxL) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_kv_compact: L %d > %d", L, kMaxL);
+    if (dt != DDTREE_F32 && dt != DDTREE_BF16) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_kv_compact: unknown dtype %d", dt);
+    const int64_t row_bytes = static_cast<int64_t>(Hkv) * d * elem_size(dt);
+    if (row_bytes % 16 || row_bytes > (1 << 24))
+        return fail(DDTREE_ERR_UNSUPPORTED, "ddtree_kv_compact: a K/V row (%lld bytes) must be a multiple of 16 bytes",
+                    static_cast<long long>(row_bytes));
+    if (!k_tree || !v_tree || !k_cache || !v_cache || !dst_row || !accept_len || !accept_nodes)
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_kv_compact: a required pointer is NULL");
+    for (int l = 0; l < layers; ++l) {
+        if (!k_tree[l] || !v_tree[l] || !k_cache[l] || !v_cache[l])
+            return fail(DDTREE_ERR_INVALID_ARG, "ddtree_kv_compact: layer %d has a NULL buffer", l);
+        if (!aligned16(k_tree[l]) || !aligned16(v_tree[l]) || !aligned16(k_cache[l]) || !aligned16(v_cache[l]))
+            return fail(DDTREE_ERR_INVALID_ARG, "ddtree_kv_compact: layer %d: buffers must be 16-byte aligned", l);
+    }
+    const cudaError_t e = launch_kv_compact(R, B + 1, L, static_cast<int>(row_bytes), layers, k_tree, v_tree, k_cache, v_cache,
+                                            dst_row, accept_len, accept_nodes, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_kv_compact: %s", cudaGetErrorString(e));
+    return DDTREE_OK;
+}
+
 static int fill_attn_args(const char* fn, AttnArgs& a, const void* q, const void* k_cache, const void* v_cache,
                           const int32_t* cu_prefix_host, const int32_t* cu_prefix, const void* k_tree,
                           const void* v_tree, const uint32_t* anc_mask, const int32_t* n_rows, void* out, float* lse,

@@ -67,6 +67,12 @@ struct AttnArgs {
 };
 cudaError_t launch_tree_attention_f32(const AttnArgs& a, cudaStream_t st);
 
+constexpr int kCompactLayersPerLaunch = 64;  // pointer tables travel as kernel parameters (4 x 64 x 8 bytes)
+cudaError_t launch_kv_compact(int R, int N, int L, int row_bytes, int layers, const void* const* k_tree,
+                              const void* const* v_tree, void* const* k_cache, void* const* v_cache,
+                              const int64_t* dst_row, const int32_t* accept_len, const int32_t* accept_nodes,
+                              cudaStream_t st);
+
 size_t tree_attention_bf16_workspace(const AttnArgs& a, const int32_t* cu_prefix_host);
 // Returns a ddtree_status (descriptor creation can fail with its own message).
 int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host, void* ws, size_t ws_bytes,

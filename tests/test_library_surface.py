@@ -56,3 +56,12 @@ def test_validation_without_gpu(lib):
     assert lib.ddtree_build(p, 7, 8, 1, 1, 8, 2, 1, *none, None, 0, None) == 1  # bad dtype
     assert lib.ddtree_build(p + 4, 0, 8, 1, 1, 8, 2, 1, *none, None, 0, None) == 1  # misaligned
     assert lib.ddtree_accept(p, 0, 8, 1, 1, 8, 1, *([None] * 8), None, 0, None) == 1  # null outputs
+    # ddtree_kv_compact: every refusal happens on the host, before any launch
+    ptrs = (ctypes.c_void_p * 2)(p, p)
+    assert lib.ddtree_kv_compact(1, 8, 4, 2, 64, 1, 2, None, ptrs, ptrs, ptrs, p, p, p, None) == 1       # NULL table
+    assert lib.ddtree_kv_compact(1, 8, 4, 1, 4, 1, 2, ptrs, ptrs, ptrs, ptrs, p, p, p, None) == 2        # 8-byte rows
+    assert b"multiple of 16" in lib.ddtree_last_error()
+    bad = (ctypes.c_void_p * 2)(p, p + 4)
+    assert lib.ddtree_kv_compact(1, 8, 4, 2, 64, 1, 2, ptrs, bad, ptrs, ptrs, p, p, p, None) == 1        # misaligned layer buffer
+    assert lib.ddtree_kv_compact(1, 8, 4, 2, 64, 9, 2, ptrs, ptrs, ptrs, ptrs, p, p, p, None) == 1       # bad dtype
+    assert lib.ddtree_kv_compact(1, 8, 4, 2, 64, 1, 0, ptrs, ptrs, ptrs, ptrs, p, p, p, None) == 1       # no layers
