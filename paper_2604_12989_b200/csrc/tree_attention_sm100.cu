@@ -742,12 +742,21 @@ combine_kernel(const KernelParams p) {
     const int h = static_cast<int>(task % p.Hq);
     const int node = static_cast<int>((task / p.Hq) % p.N);
     const int r = static_cast<int>(task / (static_cast<long long>(p.Hq) * p.N));
-    if (node >= p.n_rows[r]) return;
     const int kvh = h / p.G, grow = node * p.G + h % p.G;
     const size_t split_stride = static_cast<size_t>(p.R) * p.Hkv * p.rows_pad;
     const size_t row0 = (static_cast<size_t>(r) * p.Hkv + kvh) * p.rows_pad + grow;
+    // One round trip to L2 for everything this row needs: the row count of the request, the (max, sum)
+    // pairs and the rows of up to 8 splits are requested together, before any of them is looked at
+    // (rows of padding nodes and of empty splits lie inside the buffer; their contents are never used).
+    const __half* po = p.part_o + row0 * kTile + lane * 4;
+    const int n_r = p.n_rows[r];
     float2 ml = make_float2(-CUDART_INF_F, 0.f);
     if (lane < p.splits) ml = p.part_ml[lane * split_stride + row0];
+    uint2 raw[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+        raw[u] = u < p.splits ? *reinterpret_cast<const uint2*>(po + u * split_stride * kTile) : make_uint2(0u, 0u);
+    if (node >= n_r) return;
     float M = ml.y > 0.f ? ml.x : -CUDART_INF_F;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
@@ -757,17 +766,18 @@ combine_kernel(const KernelParams p) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(kFull, l, o);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    const __half* po = p.part_o + row0 * kTile + lane * 4;
-#pragma unroll 4
-    for (int s = 0; s < p.splits; ++s) {
+    auto add = [&](int s, uint2 v) {
         const float ws = __shfl_sync(kFull, wl, s);
-        if (ws == 0.f) continue;  // warp-uniform
-        const uint2 raw = *reinterpret_cast<const uint2*>(po + s * split_stride * kTile);
-        const float2 o01 = __half22float2(*reinterpret_cast<const __half2*>(&raw.x));
-        const float2 o23 = __half22float2(*reinterpret_cast<const __half2*>(&raw.y));
+        if (ws == 0.f) return;  // warp-uniform
+        const float2 o01 = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+        const float2 o23 = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
         acc[0] = fmaf(ws, o01.x, acc[0]); acc[1] = fmaf(ws, o01.y, acc[1]);
         acc[2] = fmaf(ws, o23.x, acc[2]); acc[3] = fmaf(ws, o23.y, acc[3]);
-    }
+    };
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+        if (u < p.splits) add(u, raw[u]);
+    for (int s = 8; s < p.splits; ++s) add(s, *reinterpret_cast<const uint2*>(po + s * split_stride * kTile));
     const float inv = 1.f / l;
     const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv);
     const __nv_bfloat162 b1 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
