@@ -34,8 +34,8 @@ METRIC = "ddtree_verify_rounds_per_s"
 UNIT = "rounds/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of tree_attention_bf16_kernel on the
-# benchmark workload, from the ncu capture summarised in profiles/tree_attention_bf16_config1.txt.
-NCU_TRAFFIC_BYTES = {1: 17657344, 2: 74303232}
+# workload, from the ncu captures summarised in profiles/tree_attention_bf16_config{1,2}.txt.
+NCU_TRAFFIC_BYTES = {1: 17653504, 2: 74303232}
 
 
 def peaks():
