@@ -23,6 +23,7 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
+#include <algorithm>
 #include <mutex>
 #include <unordered_map>
 #include <vector>
@@ -45,6 +46,7 @@ constexpr uint32_t kColO = 256;       // O accumulators of the two column halves
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kMaxOrdered = 128;
 constexpr uint32_t kErrTimeout = 0x5101;
 constexpr uint32_t kErrAlign = 0x5102;
 
@@ -254,6 +256,10 @@ struct KernelParams {
     uint32_t* status;
     int R, N, W, Hq, Hkv, G, splits, rows_pad;
     float scale_log2;
+    // blockIdx.z -> request, longest prefix first (CTAs are dispatched in index order: the long ones must
+    // not be left for the end); identity when the batch has more than kMaxOrdered requests
+    int ordered;
+    uint16_t order[kMaxOrdered];
 };
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -311,7 +317,7 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     pdl_wait();               // everything read below may come from the previous kernel of the stream
     const int split = blockIdx.x;
     const int kvh = blockIdx.y % p.Hkv, rt = blockIdx.y / p.Hkv;
-    const int r = blockIdx.z;
+    const int r = p.ordered ? p.order[blockIdx.z] : blockIdx.z;
     const int n = min(p.n_rows[r], p.N);
     if (rt * kTile >= n * p.G) return;  // whole row tile is padding
     const int p0 = p.cu_prefix[r], P = p.cu_prefix[r + 1] - p0;
@@ -902,7 +908,7 @@ extern "C" int ddtree_debug_set_trace(void* device_buffer) {
 }
 #endif
 
-int launch_tree_attention_bf16(const AttnArgs& a, const int32_t*, void* ws, size_t, cudaStream_t st) {
+int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host, void* ws, size_t, cudaStream_t st) {
     const Plan pl = make_plan(a);
     CUtensorMap mq, mkc, mvc, mkt, mvt;
     const uint64_t tree_rows = static_cast<uint64_t>(a.R) * a.N;
@@ -927,6 +933,16 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t*, void* ws, size
     p.R = a.R; p.N = a.N; p.W = a.W; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = a.G;
     p.splits = pl.splits; p.rows_pad = pl.rows_pad;
     p.scale_log2 = a.scale * kLog2e;
+    p.ordered = 0;
+    if (cu_prefix_host && a.R > 1 && a.R <= kMaxOrdered) {
+        std::vector<int> idx(a.R);
+        for (int i = 0; i < a.R; ++i) idx[i] = i;
+        std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) {
+            return cu_prefix_host[x + 1] - cu_prefix_host[x] > cu_prefix_host[y + 1] - cu_prefix_host[y];
+        });
+        for (int i = 0; i < a.R; ++i) p.order[i] = static_cast<uint16_t>(idx[i]);
+        p.ordered = 1;
+    }
 
     static const size_t smem_bytes = sizeof(Smem);
     static_assert(sizeof(Smem) <= 232448, "exceeds the 227 KB of shared memory a CTA may opt in to");
