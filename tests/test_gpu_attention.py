@@ -256,3 +256,24 @@ def test_bf16_workspace_too_small_is_refused():
                                  att.cu_prefix.tolist(), torch.from_numpy(att.cu_prefix).cuda(),
                                  kt[..., :64].contiguous(), vt[..., :64].contiguous(), mask, n_rows)
     assert e.value.status == 2
+
+
+@pytest.mark.parametrize("seed", range(14))
+def test_bf16_random_shapes(seed):
+    """Random small problems: batch size, budget, group size, prefix lengths (zero, a few keys, ragged
+    ends of a 128-key tile, several tiles so that the KV range is split) and trees smaller than the
+    budget, all rows against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    R = int(rng.integers(1, 5))
+    G = int(rng.choice([1, 2, 4, 8, 16]))
+    Hkv = int(rng.choice([1, 2])) if G >= 8 else int(rng.choice([1, 2, 4]))
+    B = int(rng.choice([1, 2, 7, 31, 32, 33, 63, 64, 100, 129, 200, 300]))
+    kinds = [0, int(rng.integers(1, 8)), 127, 128, 129, int(rng.integers(130, 700)), int(rng.integers(700, 2600))]
+    prefix = tuple(int(rng.choice(kinds)) for _ in range(R))
+    L = int(rng.integers(2, 9))
+    K = int(rng.integers(1, 5))
+    w, att, trees = bf16_case(R, B, G * Hkv, Hkv, prefix, K=K, L=L, seed=seed)
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse)
+    for r in range(R):
+        assert (out[r, trees[r].n_rows:] == 0).all()  # rows past the tree are left alone
