@@ -113,7 +113,8 @@ int ddtree_build(const void* drafter_logits, int dt, int64_t row_stride_elems,
  * Inputs
  *   q                [R, B+1, Hq, d]
  *   k_cache, v_cache [sum P, Hkv, d]      d contiguous
- *   cu_prefix_host   [R+1] int32 HOST     exclusive prefix sums of the P_r (used for planning)
+ *   cu_prefix_host   [R+1] int32 HOST     exclusive prefix sums of the P_r (used for planning: KV splits,
+ *                                         workspace size, longest-first dispatch of the requests)
  *   cu_prefix        [R+1] int32 device   the same values on the device
  *   k_tree, v_tree   [R, B+1, Hkv, d]     this round's K/V of the tree rows (not yet in the cache)
  *   anc_mask         [R, B+1, W] uint32, n_rows [R] int32   as written by ddtree_build
@@ -121,7 +122,8 @@ int ddtree_build(const void* drafter_logits, int dt, int64_t row_stride_elems,
  *   out              [R, B+1, Hq, d]      same element type as q; rows >= n_rows[r] are left untouched
  *   lse_or_null      [R, B+1, Hq] fp32    optional natural-log sum of exp(scaled scores)
  * dt = DDTREE_BF16: bf16 inputs, fp32 accumulation on the tensor cores, probabilities rounded to
- *   bf16 before the PV product; requires d == 128.  dt = DDTREE_F32: fp32 FMA arithmetic; d in
+ *   bf16 before the PV product (when the KV range of a request is split over several CTAs, each
+ *   part's normalised rows pass through fp16 before they are merged); requires d == 128.  dt = DDTREE_F32: fp32 FMA arithmetic; d in
  *   {64, 128}.  Hq must be a multiple of Hkv with Hq/Hkv in {1, 2, 4, 8, 16}.
  * softmax_scale 0 means 1/sqrt(d).  All tensors must be 16-byte aligned.
  * workspace: at least ddtree_tree_attention_workspace_bytes(...) bytes, 16-byte aligned.
