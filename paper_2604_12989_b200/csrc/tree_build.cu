@@ -25,6 +25,9 @@ __device__ __forceinline__ unsigned orderable(float f) {
     const unsigned u = __float_as_uint(f);
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
+__device__ __forceinline__ float from_orderable(unsigned k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 
 // Sorted list of the best entries seen by a warp: lane k holds the k-th best (value, id).
 struct WarpTopK {
@@ -252,42 +255,77 @@ tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restric
         int bests = lane == 0 ? 0 : -1;
         const unsigned none = orderable(-CUDART_INF_F);
         __syncwarp();
+#ifdef DDTREE_TRACE
+        long long ps[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#define PSTAMP(i) do { if (t == 20) { long long t_; asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_)); ps[i] = t_; } } while (0)
+#else
+#define PSTAMP(i) ((void)0)
+#endif
         for (int t = 0; t < B; ++t) {
+            PSTAMP(0);
             const unsigned key = orderable(bestv);
             const unsigned mx = __reduce_max_sync(kFull, key);
             if (mx == none) break;  // heap empty: fewer than B prefixes exist in S_K
             const int src = __ffs(__ballot_sync(kFull, key == mx)) - 1;
             const int u = __shfl_sync(kFull, bests, src);
-            const float v = __shfl_sync(kFull, bestv, src);
+            const float v = from_orderable(mx);  // the winning candidate's score
+            PSTAMP(1);
             const int du = sh.depth[u], cu = sh.cc[u];
             const float su = sh.sigma[u];
             const int n = count++;
+            // This lane's best among its slots other than u (slot s sits on lane s % 32; n is not written
+            // yet).  These reads depend on nothing the pop computes, so they travel with the reads of
+            // u's state; the two slots that change are patched in from registers below.  The trip count
+            // is the same for every lane: a loop that lanes leave at different times costs the warp
+            // about 150 cycles per pop.
+            bestv = -CUDART_INF_F; bests = -1;
+            auto look = [&](int i) {
+                const int j = i * 32 + lane;
+                const float cj = sh.cand[min(j, n - 1)];
+                const float c = ((j < n) & (j != u)) ? cj : -CUDART_INF_F;
+                const bool up = c > bestv;
+                bestv = up ? c : bestv;
+                bests = up ? j : bests;
+            };
+            if (B < 128) {  // at most 4 slots per lane: straight-line code, the reads leave together
+#pragma unroll
+                for (int i = 0; i < 4; ++i) look(i);
+            } else {
+                const int trips = (n + 31) >> 5;
+#pragma unroll 4
+                for (int i = 0; i < trips; ++i) look(i);
+            }
+            PSTAMP(2);
             const float cand_u = (cu + 1 < K) ? su + sh.logq[du * K + cu + 1] : -CUDART_INF_F;
             const float cand_n = (du + 1 < L) ? v + sh.logq[(du + 1) * K] : -CUDART_INF_F;
-            __syncwarp();  // all lanes have read u's state before lane 0 overwrites it
-            if (lane == 0) {
-                sh.parent[n] = static_cast<short>(u);
-                sh.rank[n] = static_cast<unsigned char>(cu + 1);
-                sh.depth[n] = static_cast<unsigned char>(du + 1);
-                sh.sigma[n] = v;
-                sh.cc[n] = 0;
-                sh.cc[u] = static_cast<unsigned char>(cu + 1);
-                sh.cand[u] = cand_u;
-                sh.cand[n] = cand_n;
+            // ties go to the lowest slot, as in a scan over the slots in ascending order
+            const bool take_u = (lane == (u & 31)) & ((cand_u > bestv) | ((cand_u == bestv) & (u < bests)));
+            bestv = take_u ? cand_u : bestv;
+            bests = take_u ? u : bests;
+            const bool take_n = (lane == (n & 31)) & (cand_n > bestv);
+            bestv = take_n ? cand_n : bestv;
+            bests = take_n ? n : bests;
+            PSTAMP(3);
+            __syncwarp();  // all lanes have read u's state and their slots before lane 0 overwrites them
+            {   // lane 0 writes; the other lanes store the same values to a spare slot instead of branching
+                const int wn = lane == 0 ? n : kSlots - 1, wu = lane == 0 ? u : kSlots - 1;
+                sh.parent[wn] = static_cast<short>(u);
+                sh.rank[wn] = static_cast<unsigned char>(cu + 1);
+                sh.depth[wn] = static_cast<unsigned char>(du + 1);
+                sh.sigma[wn] = v;
+                sh.cc[wn] = 0;
+                sh.cand[wn] = cand_n;
+                sh.cc[wu] = static_cast<unsigned char>(cu + 1);
+                sh.cand[wu] = cand_u;
             }
             __syncwarp();
-            if (lane == (u & 31)) {  // this lane's best was consumed: rescan its slots
-                bestv = -CUDART_INF_F; bests = -1;
-                for (int j = lane; j < count; j += 32) {
-                    const float c = sh.cand[j];
-                    if (c > bestv) { bestv = c; bests = j; }
-                }
-            } else if (lane == (n & 31)) {
-                if (cand_n > bestv) { bestv = cand_n; bests = n; }
-            }
+            PSTAMP(4);
         }
         __syncwarp();
         BTRACE(3);
+#ifdef DDTREE_TRACE
+        if (g_build_trace && blockIdx.x == 0 && lane == 0) for (int i = 0; i < 5; ++i) g_build_trace[8 + i] = ps[i];
+#endif
 
         // ---- 3. level order: rows sorted by (depth, parent row, rank) --------------------------
         for (int j = lane; j < count; j += 32) atomicAdd(&sh.lvl_cnt[sh.depth[j]], 1);
