@@ -15,6 +15,8 @@
 //   warp 9     MMA issuer: S = Q K^T (operands in shared memory) runs one tile ahead into two TMEM
 //              score buffers; O_h += P_h V_h (P read from TMEM, V as an MN-major shared-memory
 //              operand) as soon as half h of the tile is ready; owns the TMEM allocation
+// A last row tile of at most 16 rows (the root's G rows of a tree of 2^k nodes) takes a path of its own
+// in batches that fill the SMs several times over: see tail_tile_cta.
 // The ancestor bitmask is applied only on tree tiles; prefix tiles need at most a length test on
 // the request's last tile.  Each split writes its normalised rows (fp16) with their reference maximum
 // and sum; a combine kernel merges them by log-sum-exp.  Every wait is bounded: when one gives up, the CTA raises a flag in the
@@ -176,6 +178,23 @@ __device__ __forceinline__ void umma_ts(uint32_t d, uint32_t a, uint64_t b, uint
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], " DDTREE_S32 ";" ::"r"(taddr), DDTREE_W32(v, o) : "memory")
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// 16 consecutive columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t (&v)[16], uint32_t taddr) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                 : "r"(taddr));
+}
+// Named barriers of the short-tile path: id 1 + g over the 128 threads of key group g (plain and with an
+// OR vote), id 3 over both groups.
+__device__ __forceinline__ void bar_keys(int g) { asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory"); }
+__device__ __forceinline__ bool bar_keys_or(int g, bool x) {
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %2, 0;\n\tbar.red.or.pred p, %1, 128, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(r) : "r"(1 + g), "r"(static_cast<uint32_t>(x)) : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ void bar_all_keys() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart.
 //   K-major operand (Q, K): rows of 64 bf16 (128 bytes); the leading-dimension field is unused.
@@ -219,7 +238,10 @@ __device__ __forceinline__ void trace_clk(int idx) {
 #define TRACE_CLK(idx) trace_clk(idx)
 // Low-overhead time stamps: clock64 into registers for two steady-state tiles, written out once
 // after the loop (a stamp that writes to global memory costs ~300 cycles and distorts the loop).
-constexpr int kStampTile = 8;
+#ifndef DDTREE_STAMP_TILE
+#define DDTREE_STAMP_TILE 8
+#endif
+constexpr int kStampTile = DDTREE_STAMP_TILE;
 #define STAMP_DECL long long stamp_[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
 #define STAMP(cond, i) do { if (cond) { long long t_; asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_)); stamp_[i] = t_; } } while (0)
 #define STAMP_FLUSH(cond, base) do { if ((cond) && g_trace) { \
@@ -303,10 +325,422 @@ __device__ __forceinline__ void mask32(uint32_t (&sv)[64], int o, uint32_t word)
         if (!((word >> c) & 1u)) sv[o + c] = 0xff800000u;
 }
 
+// ---- short last row tile ----------------------------------------------------------------------
+// A tree of B = 2^k nodes plus the root leaves G rows over for a last row tile of their own; run
+// through the path below, that tile would cost as much as a full one (a fifth of all CTAs for B = 128,
+// G = 4).  With so few rows the roles of
+// rows and keys are swapped for the scores: S^T = K Q^T puts the 128 keys of a tile on the TMEM lanes
+// and the (at most 16) rows on the columns, so a thread exponentiates 16 values per tile instead of
+// 64, keeps its own partial row sums, and the tile costs little more than the copy of its K/V.  The
+// second product is swapped as well: O^T += V^T P^T with the V tile as the 128-row (MN-major) operand
+// and P^T, 16 rows x 128 keys written to shared memory by the key threads, as the narrow one; O^T
+// has the head dimension on the lanes and one column per row.  A row's reference maximum is set by
+// an exact reduction over the key threads on the first tile and whenever an exponential exceeds
+// 2^24; otherwise the threads only meet at one barrier per tile.  Two groups of 128 key threads take
+// alternate tiles, each with its own reference maxima, sums and O^T, merged at the end.  The CTA sees
+// the whole KV range of its rows (the path is used only where there are no KV splits) and writes the
+// output itself.  Measured: ~1200 cycles per KV tile against ~2200 on the full-tile path; the tensor
+// pipe is the limit (16 instructions per tile that each stream a 4 KB operand from shared memory).
+constexpr int kTailRows = 16;
+constexpr int kTailKStages = 3, kTailVStages = 3;
+constexpr uint32_t kTailQHalf = kTailRows * 128;  // one 64-wide half of the 16-row Q or P^T tile
+constexpr int kTailSBufs = 4;    // S^T = K Q^T runs four tiles ahead of the key threads
+constexpr uint32_t kColST = 0;  // S^T buffers at columns 0, 32, 64 and 96
+constexpr uint32_t kColOT = 256; // O^T of key group g at column 256 + 32 g
+
+struct TailSmem {
+    uint8_t k[kTailKStages][kTileBytes];
+    uint8_t v[kTailVStages][kTileBytes];
+    uint8_t q[2 * kTailQHalf];      // the tile's 16 query rows
+    uint8_t pt[2][2][2 * kTailQHalf];  // [group][buffer] P^T: [row][key], two 64-key halves, 128-byte swizzle (K-major operand)
+    uint64_t q_full, k_full[kTailKStages], k_free[kTailKStages], v_full[kTailVStages], v_free[kTailVStages];
+    // One barrier per buffer, each watched by one key group only: a parity wait must see every phase in turn.
+    uint64_t s_full[kTailSBufs], p_ready[2][2], o_done[2][2];
+    float red[2][4][kTailRows];  // [group][warp]: row maxima inside the loop, row sums at the end
+    float mref[2][kTailRows];    // the groups' reference maxima, exchanged at the end
+    uint32_t tmem_base;
+    uint32_t abort;
+    uint32_t key_fail[2];  // per group: a key thread's wait gave up (written before, read after a barrier of the group)
+};
+
+__device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const CUtensorMap* map_kc, const CUtensorMap* map_vc,
+                                              const CUtensorMap* map_kt, const CUtensorMap* map_vt, const KernelParams& p,
+                                              uint8_t* smem_raw, int kvh, int rt, int r, int n) {
+    TailSmem& sm = *reinterpret_cast<TailSmem*>(smem_raw);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rows = min(n * p.G - rt * kTile, kTailRows);  // valid rows of this tile (> 0: checked by the caller)
+    const int p0 = p.cu_prefix[r], P = p.cu_prefix[r + 1] - p0;
+    const int prefix_tiles = (P + kTile - 1) / kTile, tree_tiles = (n + kTile - 1) / kTile;
+    const int my_tiles = prefix_tiles + tree_tiles;  // the whole KV range (this path runs without KV splits), >= 1
+    constexpr int t_begin = 0;
+
+    volatile uint32_t* abort_flag = &sm.abort;
+    if (tid == 0) TRACE(60);
+    int k_issued = 0, v_issued = 0;
+    auto tile_row = [&](int j, bool& in_prefix) {
+        const int t = t_begin + j;
+        in_prefix = t < prefix_tiles;
+        return in_prefix ? p0 + t * kTile : r * p.N + (t - prefix_tiles) * kTile;
+    };
+    auto load_k = [&](int j) {
+        bool in_prefix;
+        const int row = tile_row(j, in_prefix), s = j % kTailKStages;
+        mbar_expect_tx(smem_u32(&sm.k_full[s]), kTileBytes);
+        for (int h = 0; h < 2; ++h)
+            tma_load_3d(smem_u32(sm.k[s]) + h * kHalfBytes, in_prefix ? map_kc : map_kt, smem_u32(&sm.k_full[s]), h * 64, kvh, row);
+    };
+    auto load_v = [&](int j) {
+        bool in_prefix;
+        const int row = tile_row(j, in_prefix), s = j % kTailVStages;
+        mbar_expect_tx(smem_u32(&sm.v_full[s]), kTileBytes);
+        for (int h = 0; h < 2; ++h)
+            tma_load_3d(smem_u32(sm.v[s]) + h * kHalfBytes, in_prefix ? map_vc : map_vt, smem_u32(&sm.v_full[s]), h * 64, kvh, row);
+    };
+    if (warp == kProducerWarp && lane == 0) {
+        mbar_init(smem_u32(&sm.q_full), 1);
+        for (int s = 0; s < kTailKStages; ++s) { mbar_init(smem_u32(&sm.k_full[s]), 1); mbar_init(smem_u32(&sm.k_free[s]), 1); }
+        for (int s = 0; s < kTailVStages; ++s) { mbar_init(smem_u32(&sm.v_full[s]), 1); mbar_init(smem_u32(&sm.v_free[s]), 1); }
+        for (int b = 0; b < kTailSBufs; ++b) mbar_init(smem_u32(&sm.s_full[b]), 1);
+        for (int b = 0; b < 4; ++b) { mbar_init(smem_u32(&sm.p_ready[0][0]) + 8 * b, 1); mbar_init(smem_u32(&sm.o_done[0][0]) + 8 * b, 1); }
+        sm.abort = 0;
+        sm.key_fail[0] = 0;
+        sm.key_fail[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const int nodes_per_tile = kTile / p.G;
+        mbar_expect_tx(smem_u32(&sm.q_full), 2 * kTailQHalf);
+        for (int h = 0; h < 2; ++h)
+            tma_load_4d(smem_u32(sm.q) + h * kTailQHalf, map_qt, smem_u32(&sm.q_full), h * 64, 0, kvh, r * p.N + rt * nodes_per_tile);
+        for (; k_issued < my_tiles && k_issued < kTailKStages; ++k_issued) load_k(k_issued);
+        for (; v_issued < my_tiles && v_issued < kTailVStages; ++v_issued) load_v(v_issued);
+    }
+    if (warp == kMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
+                     "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid < 256) {  // P^T starts as zeros; rows beyond the valid ones are never written
+        uint4* z = reinterpret_cast<uint4*>(sm.pt);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) z[tid + 256 * u] = make_uint4(0u, 0u, 0u, 0u);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    if (warp == kProducerWarp) {
+        if (lane == 0) {
+            // the two rings are polled independently: a copy starts as soon as its slot is free
+            uint32_t idle = 0;
+            while (k_issued < my_tiles || v_issued < my_tiles) {
+                bool progressed = false;
+                if (k_issued < my_tiles &&
+                    mbar_test(smem_u32(&sm.k_free[k_issued % kTailKStages]), ((k_issued / kTailKStages) - 1) & 1)) {
+                    load_k(k_issued++);
+                    progressed = true;
+                }
+                if (v_issued < my_tiles &&
+                    mbar_test(smem_u32(&sm.v_free[v_issued % kTailVStages]), ((v_issued / kTailVStages) - 1) & 1)) {
+                    load_v(v_issued++);
+                    progressed = true;
+                }
+                if (progressed) { idle = 0; continue; }
+                __nanosleep(32);
+                if (++idle > kSpinLimit) { *abort_flag = 1; break; }
+                if ((idle & 255u) == 0 && *abort_flag) break;
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        constexpr uint32_t idesc_st = instr_desc(kTailRows, false);          // 128 keys x 16 rows, both operands K-major
+        constexpr uint32_t idesc_pv = instr_desc(kTailRows, false) | (1u << 15);  // 128 head-dim x 16 rows, V^T MN-major
+        constexpr uint32_t kQHalf = kTailQHalf >> 4;                          // second 64-wide half of Q / P^T, descriptor units
+        const uint64_t q_desc = smem_desc(smem_u32(sm.q), 16);
+        const uint64_t k_desc0 = smem_desc(smem_u32(sm.k[0]), 16);
+        const uint64_t v_desc0 = smem_desc(smem_u32(sm.v[0]), kHalfBytes);
+        const uint64_t p_desc0 = smem_desc(smem_u32(sm.pt[0][0]), 16);
+        // S^T[j % 4] = K_j Q^T: the K tile is the 128-row operand, the 16 query rows the other
+        auto issue_st = [&](int j) {
+            const int s = j % kTailKStages, b = j % kTailSBufs;
+            const uint64_t kd = k_desc0 + static_cast<uint64_t>(s) * (kTileBytes >> 4);
+            const uint32_t d_s = tmem + kColST + b * 32;
+            umma_ss<false>(d_s, kd, q_desc, idesc_st);
+            umma_ss<true>(d_s, kd + 2, q_desc + 2, idesc_st);
+            umma_ss<true>(d_s, kd + 4, q_desc + 4, idesc_st);
+            umma_ss<true>(d_s, kd + 6, q_desc + 6, idesc_st);
+            umma_ss<true>(d_s, kd + 1024, q_desc + kQHalf, idesc_st);
+            umma_ss<true>(d_s, kd + 1026, q_desc + kQHalf + 2, idesc_st);
+            umma_ss<true>(d_s, kd + 1028, q_desc + kQHalf + 4, idesc_st);
+            umma_ss<true>(d_s, kd + 1030, q_desc + kQHalf + 6, idesc_st);
+            tc_commit(smem_u32(&sm.k_free[s]));
+            tc_commit(smem_u32(&sm.s_full[b]));
+        };
+        auto wait_k = [&](int j) {
+            return __all_sync(kFull, mbar_wait(smem_u32(&sm.k_full[j % kTailKStages]), (j / kTailKStages) & 1, abort_flag));
+        };
+        bool ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.q_full), 0, abort_flag));
+        for (int j = 0; j < my_tiles && j < kTailSBufs && ok; ++j) {
+            ok = wait_k(j);
+            if (!ok) break;
+            tc_fence_after();
+            if (elect_one()) issue_st(j);
+            __syncwarp();
+        }
+        STAMP_DECL;
+        for (int j = 0; j < my_tiles && ok; ++j) {
+            // One burst per tile: O_g^T += V_j^T P_j^T, then the scores of tile j+4 into the S^T buffer the key
+            // threads have just read.  Every instruction streams a 128-row operand (4 KB) from shared
+            // memory, which takes the tensor pipe ~50 cycles whatever the other extent, so a tile costs it
+            // ~850 cycles; the barriers are tested together beforehand to keep it from draining.
+            const int s = j % kTailVStages, g = j & 1, b = (j >> 1) & 1;  // key group and its P^T buffer
+            const bool more = j + kTailSBufs < my_tiles;
+            const bool st8 = j == kStampTile;
+            STAMP(st8, 0);
+            const bool k_ok = !more || mbar_test(smem_u32(&sm.k_full[(j + kTailSBufs) % kTailKStages]), ((j + kTailSBufs) / kTailKStages) & 1);
+            const bool ready = mbar_test(smem_u32(&sm.v_full[s]), (j / kTailVStages) & 1) & k_ok &
+                               mbar_test(smem_u32(&sm.p_ready[g][b]), (j >> 2) & 1);
+            if (!__all_sync(kFull, ready)) {
+                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.v_full[s]), (j / kTailVStages) & 1, abort_flag)) &&
+                     (!more || wait_k(j + kTailSBufs)) &&
+                     __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[g][b]), (j >> 2) & 1, abort_flag));
+                if (!ok) break;
+            }
+            STAMP(st8, 1);
+            tc_fence_after();
+            const uint64_t vd = v_desc0 + static_cast<uint64_t>(s) * (kTileBytes >> 4);
+            const uint64_t pd = p_desc0 + static_cast<uint64_t>(g * 2 + b) * ((2 * kTailQHalf) >> 4);
+            const uint32_t d_o = tmem + kColOT + g * 32;
+            if (elect_one()) {
+                // 16 keys per instruction: 16 rows further in V, 32 bytes further in P^T's rows
+                if (j > 1) umma_ss<true>(d_o, vd, pd, idesc_pv);
+                else umma_ss<false>(d_o, vd, pd, idesc_pv);
+                umma_ss<true>(d_o, vd + 128, pd + 2, idesc_pv);
+                umma_ss<true>(d_o, vd + 256, pd + 4, idesc_pv);
+                umma_ss<true>(d_o, vd + 384, pd + 6, idesc_pv);
+                umma_ss<true>(d_o, vd + 512, pd + kQHalf, idesc_pv);
+                umma_ss<true>(d_o, vd + 640, pd + kQHalf + 2, idesc_pv);
+                umma_ss<true>(d_o, vd + 768, pd + kQHalf + 4, idesc_pv);
+                umma_ss<true>(d_o, vd + 896, pd + kQHalf + 6, idesc_pv);
+                tc_commit(smem_u32(&sm.o_done[g][b]));
+                tc_commit(smem_u32(&sm.v_free[s]));
+                if (more) issue_st(j + kTailSBufs);
+            }
+            __syncwarp();
+            STAMP(st8, 2);
+        }
+        STAMP_FLUSH(lane == 0, 0);
+    } else {
+        // ---- key threads: two groups of 128 (warps 0-3: even tiles, warps 4-7: odd tiles).  Thread c of a
+        //      group owns key c of its tiles and head-dim element c of the group's O^T.  A group has its own
+        //      reference maxima, sums and O^T, like the column halves of the full tiles: the groups never
+        //      talk inside the loop and are merged at the end like two KV splits. ----------------------
+        const int g = warp >> 2, c = tid & (kTile - 1);
+        const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const uint32_t o_addr = lane_addr + kColOT + g * 32;
+        const uint32_t p_off = (c >> 6) * kTailQHalf + ((c & 7) << 1);  // + row*128 + (chunk ^ row%8)*16
+        const int chunk = (c & 63) >> 3;
+        const int my_count = (my_tiles - g + 1) >> 1;  // tiles g, g+2, ... of this CTA
+        float mref[kTailRows], l_part[kTailRows];
+#pragma unroll
+        for (int i = 0; i < kTailRows; ++i) { mref[i] = -CUDART_INF_F; l_part[i] = 0.f; }
+        auto store_p = [&](int b, const float (&pv)[kTailRows]) {
+            uint8_t* base = sm.pt[g][b] + p_off;
+#pragma unroll
+            for (int i = 0; i < kTailRows; ++i)
+                if (i < rows)
+                    *reinterpret_cast<__nv_bfloat16*>(base + i * 128 + ((chunk ^ (i & 7)) << 4)) = __float2bfloat16_rn(pv[i]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        };
+        // completion of the product of this group's q-th tile (it read P^T[q % 2] and added to the group's O^T)
+        auto wait_pv = [&](int q) {
+            return __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[g][q & 1]), (q >> 1) & 1, abort_flag));
+        };
+        bool failed = false;
+        STAMP_DECL;
+        for (int q = 0; q < my_count; ++q) {
+            const int j = 2 * q + g, t = t_begin + j, b = q & 1, sb = j % kTailSBufs;
+            const bool st8 = j == kStampTile;
+            STAMP(st8, 0);
+            STAMP(j == kStampTile + 2, 8);
+            STAMP(j == kStampTile + 8, 9);
+            STAMP(q == 0, 10);
+            STAMP(q == 4, 12);
+            bool ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.s_full[sb]), (j / kTailSBufs) & 1, abort_flag));
+            STAMP(st8, 1);
+            uint32_t sv[kTailRows];
+#pragma unroll
+            for (int i = 0; i < kTailRows; ++i) sv[i] = 0u;
+            if (ok) {
+                tc_fence_after();
+                tmem_ld16(sv, lane_addr + kColST + sb * 32);
+            }
+            // which rows see my key
+            uint32_t vis = 0;
+            if (t < prefix_tiles) {
+                vis = t * kTile + c < P ? 0xffffu : 0u;
+            } else {
+                const int kn = (t - prefix_tiles) * kTile + c;
+                if (kn < n) {
+#pragma unroll
+                    for (int i = 0; i < kTailRows; ++i) {
+                        if (i < rows) {
+                            const int node = (rt * kTile + i) / p.G;
+                            const uint32_t word = p.anc_mask[(static_cast<size_t>(r) * p.N + node) * p.W + (kn >> 5)];
+                            vis |= ((word >> (kn & 31)) & 1u) << i;
+                        }
+                    }
+                }
+            }
+            tmem_wait_ld();
+            tc_fence_before();
+            STAMP(st8, 2);
+            float x[kTailRows], pv[kTailRows];
+            bool need = false;
+#pragma unroll
+            for (int i = 0; i < kTailRows; ++i) {
+                x[i] = ((vis >> i) & 1u) ? __uint_as_float(sv[i]) * p.scale_log2 : -CUDART_INF_F;
+                pv[i] = ex2(x[i] - (mref[i] == -CUDART_INF_F ? 0.f : mref[i]));
+                if (i < rows) need |= mref[i] == -CUDART_INF_F || !(pv[i] < 16777216.f);
+            }
+            STAMP(st8, 3);
+            // P^T[b] was read by the product of this group's tile q-2
+            if (ok && q > 1) ok = wait_pv(q - 2);
+            STAMP(st8, 4);
+            store_p(b, pv);
+            STAMP(st8, 5);
+            // A wait that gave up joins the vote, and the flag it left is read only after the barrier: every
+            // thread of the group takes the same way out (a thread missing at a later barrier would hang the others).
+            if (!ok) sm.key_fail[g] = 1;
+            const bool slow = bar_keys_or(g, need || !ok);
+            STAMP(st8, 6);
+            if (slow) {
+                if (*reinterpret_cast<volatile uint32_t*>(&sm.key_fail[g])) { failed = true; break; }
+#pragma unroll
+                for (int i = 0; i < kTailRows; ++i) {
+                    float mx = x[i];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, o));
+                    if (lane == 0) sm.red[g][warp & 3][i] = mx;
+                }
+                bar_keys(g);
+                bool bump_any = false;
+                float alpha[kTailRows];
+#pragma unroll
+                for (int i = 0; i < kTailRows; ++i) {
+                    const float m_tile = fmaxf(fmaxf(sm.red[g][0][i], sm.red[g][1][i]), fmaxf(sm.red[g][2][i], sm.red[g][3][i]));
+                    const bool bump = m_tile > mref[i] + 8.f;
+                    alpha[i] = bump ? ex2(mref[i] - m_tile) : 1.f;
+                    if (bump) { l_part[i] *= alpha[i]; mref[i] = m_tile; }
+                    if (i < rows) bump_any |= bump;
+                    pv[i] = ex2(x[i] - (mref[i] == -CUDART_INF_F ? 0.f : mref[i]));
+                }
+                if (q > 0 && bump_any) {  // the group's O^T holds the sum over its earlier tiles: scale its columns
+                    if (!wait_pv(q - 1)) sm.key_fail[g] = 1;
+                    tc_fence_after();
+                    uint32_t ov[kTailRows];
+                    tmem_ld16(ov, o_addr);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < kTailRows; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha[i]);
+                    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+                                 ::"r"(o_addr), "r"(ov[0]), "r"(ov[1]), "r"(ov[2]), "r"(ov[3]), "r"(ov[4]), "r"(ov[5]), "r"(ov[6]),
+                                   "r"(ov[7]), "r"(ov[8]), "r"(ov[9]), "r"(ov[10]), "r"(ov[11]), "r"(ov[12]), "r"(ov[13]), "r"(ov[14]), "r"(ov[15])
+                                 : "memory");
+                    tmem_wait_st();
+                    tc_fence_before();
+                }
+                store_p(b, pv);
+                bar_keys(g);
+                if (*reinterpret_cast<volatile uint32_t*>(&sm.key_fail[g])) { failed = true; break; }
+            }
+#pragma unroll
+            for (int i = 0; i < kTailRows; ++i) l_part[i] += pv[i];
+            if (c == 0) mbar_arrive(smem_u32(&sm.p_ready[g][b]));
+            STAMP(st8, 7);
+        }
+        STAMP(true, 11);
+        STAMP_FLUSH(c == 0, g ? 32 : 16);
+
+        // ---- epilogue: row sums over each group's threads, then group 0 merges the two groups and thread c
+        //      writes head-dim element c of every row ----------------------------------------------------
+        {
+            bool ok = !failed;
+            if (ok && my_count > 1) ok = wait_pv(my_count - 2);
+            if (ok && my_count > 0) ok = wait_pv(my_count - 1);
+            if (!ok) sm.key_fail[g] = 1;
+#pragma unroll
+            for (int i = 0; i < kTailRows; ++i) {
+                float sum = l_part[i];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(kFull, sum, o);
+                if (lane == 0) sm.red[g][warp & 3][i] = sum;
+                if (c == i) sm.mref[g][i] = mref[i];
+            }
+            tc_fence_before();
+            bar_all_keys();
+            const volatile uint32_t* kf = sm.key_fail;
+            if (g == 0 && !(kf[0] | kf[1])) {
+                tc_fence_after();
+                const bool two = my_tiles > 1;  // the other group had tiles: its O^T has been written
+                uint32_t oa[kTailRows], ob[kTailRows];
+                tmem_ld16(oa, lane_addr + kColOT);
+                if (two) tmem_ld16(ob, lane_addr + kColOT + 32);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < kTailRows; ++i) {
+                    if (i < rows) {
+                        const float l_a = sm.red[0][0][i] + sm.red[0][1][i] + sm.red[0][2][i] + sm.red[0][3][i];
+                        const float l_b = sm.red[1][0][i] + sm.red[1][1][i] + sm.red[1][2][i] + sm.red[1][3][i];
+                        const float m_a = mref[i], m_b = sm.mref[1][i];
+                        const float m_row = fmaxf(m_a, m_b);
+                        const float w_a = m_a == -CUDART_INF_F ? 0.f : ex2(m_a - m_row);
+                        const float w_b = (!two || m_b == -CUDART_INF_F) ? 0.f : ex2(m_b - m_row);
+                        const float l_row = l_a * w_a + l_b * w_b;
+                        const float f = l_row > 0.f ? 1.f / l_row : 0.f;
+                        float o = __uint_as_float(oa[i]) * (w_a * f);
+                        if (w_b > 0.f) o = fmaf(__uint_as_float(ob[i]), w_b * f, o);
+                        const int grow = rt * kTile + i, node = grow / p.G;
+                        const size_t head_row = (static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + grow % p.G;
+                        p.out[head_row * kTile + c] = __float2bfloat16_rn(o);
+                        if (c == 0 && p.lse) p.lse[head_row] = (m_row + log2f(l_row)) / kLog2e;
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown -------------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) TRACE(61);
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+    if (sm.abort) {
+        if (warp == kProducerWarp && lane == 0) {
+            uint32_t scratch = 0;
+            mbar_wait(smem_u32(&sm.q_full), 0, &scratch);
+            for (int j = max(0, k_issued - kTailKStages); j < k_issued; ++j)
+                mbar_wait(smem_u32(&sm.k_full[j % kTailKStages]), (j / kTailKStages) & 1, &scratch);
+            for (int j = max(0, v_issued - kTailVStages); j < v_issued; ++j)
+                mbar_wait(smem_u32(&sm.v_full[j % kTailVStages]), (j / kTailVStages) & 1, &scratch);
+            atomicExch(p.status, kErrTimeout);
+        }
+        __syncthreads();
+    }
+}
+
+// kShortTile: the grid's last row tile takes the short-tile path.  A kernel of its own rather than a run-time
+// flag: with that path compiled in, a layer of a one-request batch (CTAs that live ~10 us) was measured
+// ~2 us slower although none of its CTAs takes the path, and such batches never use it.
+template <bool kShortTile>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kc,
                            const __grid_constant__ CUtensorMap map_vc, const __grid_constant__ CUtensorMap map_kt,
-                           const __grid_constant__ CUtensorMap map_vt, const KernelParams p) {
+                           const __grid_constant__ CUtensorMap map_vt, const __grid_constant__ CUtensorMap map_qt,
+                           const KernelParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
     if (smem_u32(smem_raw) & 1023u) {  // the 128-byte swizzle needs 1024-byte aligned tiles
@@ -320,6 +754,12 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     const int r = p.ordered ? p.order[blockIdx.z] : blockIdx.z;
     const int n = min(p.n_rows[r], p.N);
     if (rt * kTile >= n * p.G) return;  // whole row tile is padding
+    if constexpr (kShortTile) {
+        if (rt == p.rows_pad / kTile - 1) {
+            tail_tile_cta(&map_qt, &map_kc, &map_vc, &map_kt, &map_vt, p, smem_raw, kvh, rt, r, n);
+            return;
+        }
+    }
     const int p0 = p.cu_prefix[r], P = p.cu_prefix[r + 1] - p0;
     const int prefix_tiles = (P + kTile - 1) / kTile, tree_tiles = (n + kTile - 1) / kTile;
     const int tiles = prefix_tiles + tree_tiles;
@@ -872,6 +1312,7 @@ int get_map(CUtensorMap* out, const void* base, int rank, uint64_t d1, uint64_t 
 
 struct Plan {
     int row_tiles, rows_pad, splits;
+    int tail;  // the last row tile takes the short-tile path
     size_t off_ml, total;
 };
 
@@ -890,6 +1331,11 @@ Plan make_plan(const AttnArgs& a) {
         if (s < 1) s = 1;
     }
     pl.splits = s;
+    // The short-tile path pays off where the SMs work through several CTAs each: its KV tiles cost half
+    // as much.  When all CTAs run at once (a few requests, KV splits) it does not: the data comes straight
+    // from HBM, its tiles are too short to hide that latency behind three-deep rings, and it would
+    // only finish after the full tiles' CTAs.
+    pl.tail = (base >= 148 && a.N * a.G - (pl.row_tiles - 1) * kTile <= kTailRows && kTailRows % a.G == 0) ? 1 : 0;
     const size_t rows = static_cast<size_t>(s) * a.R * a.Hkv * pl.rows_pad;
     pl.off_ml = (rows * kTile * 2 + 255) / 256 * 256;
     pl.total = pl.off_ml + (rows * 8 + 255) / 256 * 256;
@@ -910,10 +1356,12 @@ extern "C" int ddtree_debug_set_trace(void* device_buffer) {
 
 int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host, void* ws, size_t, cudaStream_t st) {
     const Plan pl = make_plan(a);
-    CUtensorMap mq, mkc, mvc, mkt, mvt;
+    CUtensorMap mq, mkc, mvc, mkt, mvt, mqt;
     const uint64_t tree_rows = static_cast<uint64_t>(a.R) * a.N;
     int rc = get_map(&mq, a.q, 4, a.G, a.Hkv, tree_rows, a.G, kTile / a.G);
     if (rc) return rc;
+    mqt = mq;  // the 16 query rows of a short last row tile
+    if (pl.tail && (rc = get_map(&mqt, a.q, 4, a.G, a.Hkv, tree_rows, a.G, kTailRows / a.G))) return rc;
     if ((rc = get_map(&mkt, a.k_tree, 3, a.Hkv, 0, tree_rows, 1, kTile))) return rc;
     if ((rc = get_map(&mvt, a.v_tree, 3, a.Hkv, 0, tree_rows, 1, kTile))) return rc;
     if (a.total_prefix > 0) {
@@ -945,6 +1393,7 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
     }
 
     static const size_t smem_bytes = sizeof(Smem);
+    static_assert(sizeof(TailSmem) <= sizeof(Smem), "the short-tile path lives in the same allocation");
     static_assert(sizeof(Smem) <= 232448, "exceeds the 227 KB of shared memory a CTA may opt in to");
     {   // opt in to the large dynamic shared-memory size once per device
         static std::mutex mu;
@@ -953,16 +1402,20 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
         cudaGetDevice(&dev);
         std::lock_guard<std::mutex> g(mu);
         if (dev < 0 || dev >= 64 || !done[dev]) {
-            const cudaError_t e = cudaFuncSetAttribute(tree_attention_bf16_kernel,
-                                                       cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                       static_cast<int>(smem_bytes));
+            cudaError_t e = cudaFuncSetAttribute(tree_attention_bf16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 static_cast<int>(smem_bytes));
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(tree_attention_bf16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem_bytes));
             if (e != cudaSuccess)
                 return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: shared memory opt-in: %s", cudaGetErrorString(e));
             if (dev >= 0 && dev < 64) done[dev] = true;
         }
     }
     dim3 grid(pl.splits, pl.row_tiles * a.Hkv, a.R);
-    cudaError_t e = launch_pdl(tree_attention_bf16_kernel, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, p);
+    cudaError_t e = pl.tail
+        ? launch_pdl(tree_attention_bf16_kernel<true>, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, mqt, p)
+        : launch_pdl(tree_attention_bf16_kernel<false>, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, mqt, p);
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: launch: %s", cudaGetErrorString(e));
     if (pl.splits > 1) {
         const long long tasks = static_cast<long long>(a.R) * a.N * a.Hq;

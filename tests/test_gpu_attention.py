@@ -149,6 +149,66 @@ def test_bf16_two_tree_tiles_and_heap_that_ran_empty():
     assert (out[1, 9:] == 0).all()  # padding rows untouched
 
 
+# A last row tile of at most 16 rows (the root's G rows left over by a tree of 2^k nodes, typically)
+# takes a path of its own when the batch fills the SMs several times over (R * Hkv * row tiles >= 148):
+# keys on the TMEM lanes, swapped products, two groups of key threads taking alternate tiles.
+# (R, B, Hq, Hkv): rows of the short tile = (B + 1) * G mod 128.
+SHORT_TILE_SHAPES = [
+    (38, 32, 8, 2),    # 4 rows
+    (50, 64, 4, 1),    # 4 rows after two full tiles
+    (40, 3, 16, 4),    # the whole problem is one short tile (16 rows) per KV head
+    (150, 1, 8, 1),    # 2 nodes x 8 heads
+    (75, 16, 8, 1),    # 8 rows
+    (75, 8, 16, 1),    # 16 rows of one node
+    (75, 35, 4, 1),    # 16 rows from 4 nodes
+    (15, 128, 8, 2),   # two tree tiles
+]
+
+
+def short_tile_prefixes(R, seed, hi=400):
+    p = [int(x) for x in np.random.default_rng(seed).integers(0, hi, R)]
+    p[:5] = [0, 128, 129, 1, 2 * 128 + 7][:R]  # no prefix (tree keys only: one tile, one key group idle), tile boundaries
+    return tuple(p)
+
+
+@pytest.mark.parametrize("R,B,Hq,Hkv", SHORT_TILE_SHAPES)
+def test_bf16_short_last_row_tile(R, B, Hq, Hkv):
+    w, att, trees = bf16_case(R, B, Hq, Hkv, short_tile_prefixes(R, B), K=4, L=8, seed=B, sentinel=True)
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse)
+
+
+def test_bf16_short_last_row_tile_partly_and_wholly_padding():
+    # B = 35, G = 4: nodes 32..35 sit in the short tile.  Trees of 34, 9 and 36 rows: half of the short
+    # tile, none of it, all of it.
+    import dataclasses
+    R = 75
+    w, att, trees = bf16_case(R, 35, 4, 1, short_tile_prefixes(R, 7, 300), K=4, L=8, seed=2)
+    assert all(t.n_rows == 36 for t in trees)
+    for r in range(0, R, 3):
+        trees[r] = dataclasses.replace(trees[r], n_rows=34)  # the first rows of a level-order tree are a tree
+    for r in range(1, R, 3):
+        trees[r] = orc.build(wl.drafter_logits(w, r, "peak", 2), 1, w.B, 0, 3)
+        assert trees[r].n_rows == 9
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse)
+    assert (out[0, 34:] == 0).all() and (out[1, 9:] == 0).all()
+
+
+@pytest.mark.parametrize("profile", ["growing", "exploding", "shrinking"])
+@pytest.mark.parametrize("R,B,prefix", [(19, 32, 6 * 128 + 17), (37, 3, 9 * 128 + 1)])
+def test_bf16_short_last_row_tile_scores_that_outgrow_the_reference_maximum(profile, R, B, prefix):
+    # as the test of that name for the full tiles: here the reference maximum is shared by the 128 key
+    # threads of a group and the accumulated O^T has to be rescaled when it moves
+    w, att, trees = bf16_case(R, B, 16, 4, (prefix,) * R, seed=13)
+    k = wl.bf16_to_f64(att.k_cache).astype(np.float32)
+    tiles = (np.arange(k.shape[0]) % prefix) // 128
+    factor = {"growing": 1.0 + 6.0 * tiles, "exploding": 1.0 + 40.0 * tiles, "shrinking": 40.0 / (1.0 + 6.0 * tiles)}[profile]
+    att.k_cache = wl.f32_to_bf16_bits(k * factor[:, None, None].astype(np.float32))
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse, rows_heads=[[(i, h) for i in range(trees[r].n_rows) for h in ((r % 16), 15 - (r % 16))] for r in range(R)])
+
+
 def test_bf16_many_requests_direct_path_and_repeatability():
     # R * Hkv * row_tiles >= number of SMs: no KV split, outputs written directly
     prefix = tuple(int(x) for x in np.random.default_rng(1).integers(1, 400, 40))
