@@ -277,6 +277,74 @@ def accept_walk(token: np.ndarray, parent: np.ndarray, n_rows: int, choice: np.n
     return Acceptance(len(path), path, [int(token[j]) for j in path], int(choice[cur]))
 
 
+# --------------------------------------------------------------------------
+# Section 4.4: verification walk (temperature-based sampling rule)
+# --------------------------------------------------------------------------
+#
+# "Verification then follows the target model's own decoding rule, whether greedy
+# or temperature-based sampling": at temperature T > 0 the target's choice at a
+# row is a token drawn from softmax(t / T).  The paper does not say how the draw
+# is made.  For the draw to be a function of its inputs that two programs can
+# agree on bit for bit, it is defined here as an inverse-CDF draw in token order
+# over fixed-point weights:
+#   * the random input is one 32-bit integer k per row, u = k / 2^32;
+#   * weight of token v: W_v = floor(2^40 * e_v) with e_v = 2^((x_v - max x) * c),
+#     c = float32(log2(e) / T), evaluated in float32 with one rounding per operation:
+#     t = (x_v - max) * c; n = floor(t); f = t - n; p(f) = a degree-5 polynomial for 2^f on
+#     [0, 1) in Horner form (multiply, then add); e_v = p(f) * 2^n; tokens with t < -40 get 0;
+#   * the draw is the smallest v whose inclusive prefix sum of W exceeds floor(total * k / 2^32).
+# Integer sums do not depend on the order of summation, so a parallel program gets the same token.
+# The weights differ from softmax(t / T) by less than 3e-7 relative (pinned in the tests).
+
+SAMPLING_POLY = (np.float32(0.693152487), np.float32(0.240152806), np.float32(0.0558359288),
+                 np.float32(0.00897337869), np.float32(0.00188529748))  # coefficients of f^1 .. f^5
+
+
+def sampling_weights(row: np.ndarray, temperature: float) -> List[int]:
+    """Fixed-point weights W_v of one row of target logits at temperature T (see above)."""
+    f32 = np.float32
+    x = np.asarray(row, f32)
+    c = f32(1.4426950408889634 / float(temperature))
+    with np.errstate(invalid="ignore", over="ignore"):
+        t = (x - x.max()).astype(f32) * c                 # float32 subtract, float32 multiply
+        t = t.astype(f32)
+        n = np.floor(t)
+        f = (t - n).astype(f32)
+        acc = np.full_like(f, SAMPLING_POLY[4])
+        for k in (3, 2, 1, 0):
+            acc = (acc * f).astype(f32)
+            acc = (acc + SAMPLING_POLY[k]).astype(f32)
+        acc = (acc * f).astype(f32)
+        acc = (acc + f32(1.0)).astype(f32)
+    out: List[int] = []
+    for tv, nv, pv in zip(t.tolist(), n.tolist(), acc.tolist()):
+        if not tv >= -40.0:                               # also -inf and NaN
+            out.append(0)
+            continue
+        q = int(pv * 1073741824.0)                        # p * 2^30 is an integer: p has 24 significant bits
+        out.append((q << 10) >> int(-nv))
+    return out
+
+
+def sample_token(row: np.ndarray, temperature: float, k: int) -> int:
+    """The target's choice at one row under temperature sampling with random input k in [0, 2^32)."""
+    w = sampling_weights(row, temperature)
+    total = sum(w)
+    thr = (total * int(k)) >> 32
+    acc = 0
+    for v, wv in enumerate(w):
+        acc += wv
+        if acc > thr:
+            return v
+    raise ValueError("row without a finite maximum")
+
+
+def node_sampled(target_logits: np.ndarray, temperature: float, uniforms: np.ndarray) -> np.ndarray:
+    """The target's sampled choice at every row ([rows, V] logits, one 32-bit integer per row)."""
+    return np.array([sample_token(target_logits[i], temperature, int(uniforms[i]))
+                     for i in range(target_logits.shape[0])], np.int32)
+
+
 def kv_compact(cache: np.ndarray, tree_rows: np.ndarray, prefix_len: int, path: Sequence[int]) -> np.ndarray:
     """End of a round (Section 4.4: after the walk only the accepted path stays in
     the cache): the keys (or values) of the root and of the accepted nodes are

@@ -510,3 +510,103 @@ def test_compacted_cache_is_the_context_the_last_accepted_node_saw(seed):
         np.testing.assert_allclose(out[last, h], ref[0, 0, 0].numpy(), atol=1e-12)
     for i, j in enumerate([0] + acc.nodes):
         assert ct.position_ids[j] == P + i  # cache row P + i holds the token verified at position P + i
+
+
+# --------------------------------------------------------------------------
+# Section 4.4 with the temperature-based decoding rule: fixed-point inverse-CDF draw
+# --------------------------------------------------------------------------
+
+def _exact_softmax(x, T):
+    z = (np.asarray(x, np.float64) - float(np.max(x))) / T
+    e = np.exp(z)
+    return e, e / e.sum()
+
+
+@pytest.mark.parametrize("T", [0.3, 1.0, 2.5])
+def test_sampling_weights_are_the_softmax_numerators(T):
+    rng = np.random.default_rng(5)
+    x = (rng.standard_normal(3000) * 4).astype(np.float32)
+    x[7] = -np.inf                                          # a masked token never gets weight
+    w = np.array(orc.sampling_weights(x, T), dtype=np.float64) / 2.0 ** 40
+    e, _ = _exact_softmax(x, T)
+    assert w[7] == 0 and w[int(np.argmax(x))] == 1.0        # the maximum has weight exactly 2^40
+    assert np.all(np.abs(w - e) <= 2.0 ** -40 + 5e-6 * e)
+    assert np.all(w[e < 2.0 ** -41] <= 2.0 ** -40)          # negligible tokens get (almost) nothing
+
+
+def test_sample_token_equals_the_exact_inverse_cdf_away_from_boundaries():
+    rng = np.random.default_rng(6)
+    agree = tested = 0
+    for trial in range(60):
+        V = int(rng.integers(2, 400))
+        x = (rng.standard_normal(V) * 3).astype(np.float32)
+        T = float(rng.choice([0.5, 1.0, 1.7]))
+        _, p = _exact_softmax(x, T)
+        cdf = np.cumsum(p)
+        for k in rng.integers(0, 2 ** 32, 25):
+            u = int(k) / 2.0 ** 32
+            if np.min(np.abs(cdf - u)) < 1e-5:              # the two may differ when u sits on a boundary
+                continue
+            tested += 1
+            agree += orc.sample_token(x, T, int(k)) == int(np.searchsorted(cdf, u, side="right"))
+    assert tested > 1000 and agree == tested
+
+
+def test_sample_token_on_tiny_rows_by_exact_rational_arithmetic():
+    # weights that are exact powers of two: logits k*ln2*T apart give e_v = 2^-k, no rounding anywhere
+    from fractions import Fraction
+    x = np.array([0.0, -1.0, -3.0, 0.0, -2.0], np.float32)  # with c = 1: weights 1, 1/2, 1/8, 1, 1/4
+    T = 1.4426950408889634                                   # log2(e) / T == 1.0f exactly
+    w = orc.sampling_weights(x, T)
+    assert w == [2 ** 40, 2 ** 39, 2 ** 37, 2 ** 40, 2 ** 38]
+    total = Fraction(sum(w))
+    for k in [0, 1, 2 ** 31, 2 ** 32 - 1] + [int(v) for v in np.random.default_rng(7).integers(0, 2 ** 32, 200)]:
+        u = Fraction(k, 2 ** 32)
+        acc = Fraction(0)
+        for v, wv in enumerate(w):
+            acc += Fraction(wv) / total
+            if acc > u:
+                break
+        assert orc.sample_token(x, T, k) == v
+
+
+def test_sample_token_limits_and_monotonicity():
+    rng = np.random.default_rng(8)
+    x = (rng.standard_normal(500) * 2).astype(np.float32)
+    x[:3] = -np.inf
+    x[-2:] = -200.0                                          # weight 0 at T = 1
+    assert orc.sample_token(x, 1.0, 0) == 3                  # first token with weight
+    assert orc.sample_token(x, 1.0, 2 ** 32 - 1) == 497      # last token with weight
+    ks = np.sort(rng.integers(0, 2 ** 32, 300))
+    toks = [orc.sample_token(x, 1.0, int(k)) for k in ks]
+    assert toks == sorted(toks)                              # the draw is monotone in u
+    # T -> 0: the draw is the arg-max whatever u is
+    for k in rng.integers(0, 2 ** 32, 20):
+        assert orc.sample_token(x, 1e-3, int(k)) == int(np.argmax(x))
+
+
+def test_sample_token_frequencies_follow_softmax():
+    rng = np.random.default_rng(9)
+    x = np.array([1.0, 0.0, -1.0, 2.0, 0.5, -3.0, 1.5, 0.0], np.float32)
+    T = 0.8
+    _, p = _exact_softmax(x, T)
+    n = 20000
+    counts = np.bincount([orc.sample_token(x, T, int(k)) for k in rng.integers(0, 2 ** 32, n)], minlength=8)
+    sigma = np.sqrt(n * p * (1 - p))
+    assert np.all(np.abs(counts - n * p) <= 4.5 * sigma + 1)
+
+
+def test_sampled_walk_reduces_to_the_greedy_walk_at_low_temperature():
+    rng = np.random.default_rng(10)
+    logits = rng.standard_normal((6, 50))
+    tree = orc.build(logits, 4, 20, root_token=3, prefix_len=11)
+    target = (rng.standard_normal((tree.n_rows, 50)) * 2).astype(np.float32)
+    for i in range(tree.n_rows):                             # make the target agree with some child now and then
+        kids = [j for j in range(tree.n_rows) if tree.parent[j] == i]
+        if kids and i % 2 == 0:
+            target[i, tree.token[kids[0]]] = 9.0
+    greedy = orc.accept_walk(tree.token, tree.parent, tree.n_rows, orc.node_argmax(target))
+    ks = rng.integers(0, 2 ** 32, tree.n_rows)
+    cold = orc.accept_walk(tree.token, tree.parent, tree.n_rows, orc.node_sampled(target, 1e-3, ks))
+    assert (cold.accept_len, cold.nodes, cold.bonus_token) == (greedy.accept_len, greedy.nodes, greedy.bonus_token)
+    assert greedy.accept_len >= 1
