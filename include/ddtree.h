@@ -168,6 +168,45 @@ int ddtree_accept(const void* target_logits, int dt, int64_t row_stride_elems,
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * ddtree_accept_sampled -- Section 4.4 (verifier walk under the temperature-based decoding rule:
+ * "verification follows the target model's own decoding rule, whether greedy or temperature-based
+ * sampling").  The walk is that of ddtree_accept; the target's choice at a row is a draw from
+ * softmax(target_logits[row] / temperature) instead of the arg-max.
+ *
+ * The paper does not say how the draw is made.  Here it is a function of the row, the temperature and
+ * one caller-supplied 32-bit integer per row, defined on integers so that it does not depend on the
+ * order in which anything is summed:
+ *   c    = (float)(log2(e) / (double)temperature)
+ *   W_v  = floor(2^40 * e_v),  e_v = 2^((x_v - max_v x_v) * c) evaluated in float32 with one rounding per
+ *          operation: t = (x_v - max) * c;  W_v = 0 if not t >= -40;  r = t + 12582912.0f (1.5 * 2^23: r is t
+ *          rounded to the nearest integer, ties to even, plus that constant);  n = (int)bits(r) - 0x4B400000;
+ *          f = t - (r - 12582912.0f), in [-1/2, 1/2];
+ *          p = ((((a5 f + a4) f + a3) f + a2) f + a1) f + 1  (multiply, round, add, round; a1..a5 =
+ *          0.693147004f, 0.240222424f, 0.0555073358f, 0.00967151299f, 0.00132647273f; |p / 2^f - 1| < 2e-7);
+ *          with p = sig * 2^(e - 23) (sig its 24-bit significand, e in {-1, 0}) and sh = e + 17 + n:
+ *          W_v = sig << sh if sh >= 0, else sig >> -sh   (the maximum gets exactly 2^40)
+ *   choice = smallest v with W_0 + ... + W_v > floor((sum_v W_v) * k / 2^32),  k = row_uniform[row]
+ * i.e. an inverse-CDF draw in token order with u = k / 2^32.  Supplying independent uniform k per row
+ * makes every visited row's choice an independent draw; a row's draw does not depend on the others.
+ *
+ * Inputs as for ddtree_accept, plus
+ *   temperature                      > 0 (a float: the value is used as passed)
+ *   row_uniform   [R, B+1] uint32    device memory; entries of padding rows are not read
+ * Outputs as for ddtree_accept; node_choice [R, B+1] (optional) receives the drawn token of every row,
+ * padding rows -1.  A row whose logits have no finite maximum gets choice -1 (the walk stops there).
+ * V <= 2^22.  Errors as for ddtree_accept; temperature <= 0 or not finite -> DDTREE_ERR_INVALID_ARG.
+ * ------------------------------------------------------------------------------------------ */
+size_t ddtree_accept_sampled_workspace_bytes(int R, int B, int V);
+
+int ddtree_accept_sampled(const void* target_logits, int dt, int64_t row_stride_elems,
+                          int R, int B, int V, int L,
+                          const int32_t* node_token, const int32_t* node_parent, const int32_t* n_rows,
+                          float temperature, const uint32_t* row_uniform,
+                          int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
+                          int32_t* bonus_token, int32_t* node_choice,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * ddtree_accept_static_scratch -- the paper has no counterpart; this is a packaging variant of
  * ddtree_accept for callers that cannot hand over a workspace.
  *

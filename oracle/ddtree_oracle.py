@@ -289,40 +289,48 @@ def accept_walk(token: np.ndarray, parent: np.ndarray, n_rows: int, choice: np.n
 # over fixed-point weights:
 #   * the random input is one 32-bit integer k per row, u = k / 2^32;
 #   * weight of token v: W_v = floor(2^40 * e_v) with e_v = 2^((x_v - max x) * c),
-#     c = float32(log2(e) / T), evaluated in float32 with one rounding per operation:
-#     t = (x_v - max) * c; n = floor(t); f = t - n; p(f) = a degree-5 polynomial for 2^f on
-#     [0, 1) in Horner form (multiply, then add); e_v = p(f) * 2^n; tokens with t < -40 get 0;
+#     c = float32(log2(e) / float32(T)), evaluated in float32 with one rounding per operation:
+#     t = (x_v - max) * c; n = t rounded to the nearest integer (ties to even: what adding and subtracting
+#     1.5 * 2^23 in float32 does); f = t - n, in [-1/2, 1/2]; p(f) = a degree-5 polynomial for 2^f in Horner
+#     form (multiply, then add), a float32 in [0.707, 1.415]; e_v = p(f) * 2^n taken apart into the 24-bit
+#     significand of p and a shift, so that no rounding happens after p; tokens with t < -40 get 0;
 #   * the draw is the smallest v whose inclusive prefix sum of W exceeds floor(total * k / 2^32).
 # Integer sums do not depend on the order of summation, so a parallel program gets the same token.
-# The weights differ from softmax(t / T) by less than 3e-7 relative (pinned in the tests).
+# The weights differ from the numerators of softmax(t / T) by less than 5e-6 relative (pinned in the tests).
 
-SAMPLING_POLY = (np.float32(0.693152487), np.float32(0.240152806), np.float32(0.0558359288),
-                 np.float32(0.00897337869), np.float32(0.00188529748))  # coefficients of f^1 .. f^5
+SAMPLING_POLY = (np.float32(0.693147004), np.float32(0.240222424), np.float32(0.0555073358),
+                 np.float32(0.00967151299), np.float32(0.00132647273))  # coefficients of f^1 .. f^5
+_ROUND_MAGIC = np.float32(12582912.0)  # 1.5 * 2^23: float32 addition rounds to an integer in [2^23, 2^24)
 
 
 def sampling_weights(row: np.ndarray, temperature: float) -> List[int]:
     """Fixed-point weights W_v of one row of target logits at temperature T (see above)."""
     f32 = np.float32
     x = np.asarray(row, f32)
-    c = f32(1.4426950408889634 / float(temperature))
+    c = f32(1.4426950408889634 / float(f32(temperature)))  # the temperature crosses the C boundary as a float32
     with np.errstate(invalid="ignore", over="ignore"):
-        t = (x - x.max()).astype(f32) * c                 # float32 subtract, float32 multiply
-        t = t.astype(f32)
-        n = np.floor(t)
-        f = (t - n).astype(f32)
+        t = ((x - x.max()).astype(f32) * c).astype(f32)    # float32 subtract, float32 multiply
+        live = t >= f32(-40.0)                             # false for -inf and NaN too
+        t = np.where(live, t, f32(0.0)).astype(f32)
+        r = (t + _ROUND_MAGIC).astype(f32)
+        n = r.view(np.uint32).astype(np.int64) - 0x4B400000
+        f = (t - (r - _ROUND_MAGIC).astype(f32)).astype(f32)
         acc = np.full_like(f, SAMPLING_POLY[4])
         for k in (3, 2, 1, 0):
             acc = (acc * f).astype(f32)
             acc = (acc + SAMPLING_POLY[k]).astype(f32)
         acc = (acc * f).astype(f32)
         acc = (acc + f32(1.0)).astype(f32)
+    bits = acc.view(np.uint32).astype(np.int64)
+    sig = (bits & 0x7FFFFF) | 0x800000                     # p = sig * 2^(e - 23)
+    e = (bits >> 23) - 127
     out: List[int] = []
-    for tv, nv, pv in zip(t.tolist(), n.tolist(), acc.tolist()):
-        if not tv >= -40.0:                               # also -inf and NaN
+    for ok, s_, e_, n_ in zip(live.tolist(), sig.tolist(), e.tolist(), n.tolist()):
+        if not ok:
             out.append(0)
             continue
-        q = int(pv * 1073741824.0)                        # p * 2^30 is an integer: p has 24 significant bits
-        out.append((q << 10) >> int(-nv))
+        sh = e_ + 17 + n_                                  # floor(p * 2^n * 2^40) = sig * 2^(e - 23 + n + 40)
+        out.append(s_ << sh if sh >= 0 else s_ >> -sh)
     return out
 
 

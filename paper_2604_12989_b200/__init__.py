@@ -22,6 +22,7 @@ EXPORTS = (
     "ddtree_build_workspace_bytes", "ddtree_build",
     "ddtree_tree_attention_workspace_bytes", "ddtree_tree_attention",
     "ddtree_accept_workspace_bytes", "ddtree_accept", "ddtree_accept_static_scratch",
+    "ddtree_accept_sampled_workspace_bytes", "ddtree_accept_sampled",
     "ddtree_kv_compact",
     "ddtree_device_status",
 )
@@ -63,6 +64,10 @@ def lib() -> ctypes.CDLL:
         L.ddtree_accept.argtypes = [vp, i32, i64, i32, i32, i32, i32] + [vp] * 8 + [vp, sz, vp]
         L.ddtree_accept_static_scratch.restype = i32
         L.ddtree_accept_static_scratch.argtypes = [vp, i32, i64, i32, i32, i32, i32] + [vp] * 8 + [vp]
+        L.ddtree_accept_sampled_workspace_bytes.restype = sz
+        L.ddtree_accept_sampled_workspace_bytes.argtypes = [i32] * 3
+        L.ddtree_accept_sampled.restype = i32
+        L.ddtree_accept_sampled.argtypes = [vp, i32, i64, i32, i32, i32, i32] + [vp] * 3 + [f32, vp] + [vp] * 5 + [vp, sz, vp]
         L.ddtree_kv_compact.restype = i32
         L.ddtree_kv_compact.argtypes = [i32] * 7 + [vp] * 7 + [vp]
         L.ddtree_device_status.restype = i32
@@ -198,6 +203,32 @@ def ddtree_accept(target_logits, L: int, node_token, node_parent, n_rows, worksp
         target_logits.data_ptr(), _dtype_code(target_logits), target_logits.stride(1), R, B, V, L,
         node_token.data_ptr(), node_parent.data_ptr(), n_rows.data_ptr(), out.accept_len.data_ptr(),
         out.accept_nodes.data_ptr(), out.accept_tokens.data_ptr(), out.bonus_token.data_ptr(),
+        _ptr(out.node_argmax), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return out
+
+
+def ddtree_accept_sampled(target_logits, L: int, node_token, node_parent, n_rows, temperature: float, row_uniform,
+                          workspace=None, out: Optional[Acceptance] = None, stream=None) -> Acceptance:
+    """ddtree_accept under the temperature-based decoding rule: the target's choice at a row is drawn from
+    softmax(target_logits / temperature) with the row's 32-bit random input (row_uniform: [R, B+1], an int32
+    or uint32 CUDA tensor whose bit patterns are used).  `node_argmax` of the result holds the drawn tokens."""
+    import torch
+    R, N, V = target_logits.shape
+    B = N - 1
+    assert target_logits.is_cuda and target_logits.stride(2) == 1
+    assert R == 1 or target_logits.stride(0) == N * target_logits.stride(1)
+    assert row_uniform.is_cuda and row_uniform.is_contiguous() and row_uniform.numel() == R * N and row_uniform.element_size() == 4
+    dev = target_logits.device
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=dev)
+        out = Acceptance(torch.empty(R, **i32), torch.empty(R, L, **i32), torch.empty(R, L, **i32),
+                         torch.empty(R, **i32), torch.empty(R, N, **i32))
+    if workspace is None:
+        workspace = torch.empty(max(lib().ddtree_accept_sampled_workspace_bytes(R, B, V), 256), dtype=torch.uint8, device=dev)
+    _check(lib().ddtree_accept_sampled(
+        target_logits.data_ptr(), _dtype_code(target_logits), target_logits.stride(1), R, B, V, L,
+        node_token.data_ptr(), node_parent.data_ptr(), n_rows.data_ptr(), float(temperature), row_uniform.data_ptr(),
+        out.accept_len.data_ptr(), out.accept_nodes.data_ptr(), out.accept_tokens.data_ptr(), out.bonus_token.data_ptr(),
         _ptr(out.node_argmax), workspace.data_ptr(), workspace.numel(), _stream(stream)))
     return out
 

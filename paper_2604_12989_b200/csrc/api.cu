@@ -124,9 +124,49 @@ int ddtree_accept(const void* target_logits, int dt, int64_t row_stride_elems, i
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = launch_row_argmax(target_logits, dt, row_stride_elems, R, B + 1, V, n_rows, lay, workspace, st);
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_accept: argmax pass: %s", cudaGetErrorString(e));
-    e = launch_accept_walk(R, B + 1, L, lay, workspace, node_token, node_parent, n_rows, accept_len, accept_nodes,
+    e = launch_accept_walk(R, B + 1, L, lay, workspace, nullptr, node_token, node_parent, n_rows, accept_len, accept_nodes,
                            accept_tokens, bonus_token, node_argmax, st);
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_accept: walk kernel: %s", cudaGetErrorString(e));
+    return DDTREE_OK;
+}
+
+size_t ddtree_accept_sampled_workspace_bytes(int R, int B, int V) {
+    if (R < 1 || B < 1 || B > kMaxB || V < 1) return 0;
+    return sample_layout(R * (B + 1), V).total;
+}
+
+int ddtree_accept_sampled(const void* target_logits, int dt, int64_t row_stride_elems, int R, int B, int V, int L,
+                          const int32_t* node_token, const int32_t* node_parent, const int32_t* n_rows, float temperature,
+                          const uint32_t* row_uniform, int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
+                          int32_t* bonus_token, int32_t* node_choice, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream) {
+    if (R < 1 || B < 1 || V < 1 || L < 1)
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_accept_sampled: R, B, V, L must be >= 1 (got %d %d %d %d)", R, B, V, L);
+    if (B > kMaxB) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_accept_sampled: B %d > %d", B, kMaxB);
+    if (L > kMaxL) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_accept_sampled: L %d > %d", L, kMaxL);
+    if (V > (1 << 22)) return fail(DDTREE_ERR_UNSUPPORTED, "ddtree_accept_sampled: V %d > 2^22 (64-bit weight sums)", V);
+    if (!(temperature > 0.f) || !(temperature <= 3.0e38f))
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_accept_sampled: temperature must be positive and finite");
+    const float c = static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
+    if (!(c <= 3.0e38f)) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_accept_sampled: temperature too small");
+    int rc = check_logits("ddtree_accept_sampled", target_logits, dt, row_stride_elems, V);
+    if (rc) return rc;
+    if (!node_token || !node_parent || !n_rows || !row_uniform || !accept_len || !accept_nodes || !accept_tokens || !bonus_token)
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_accept_sampled: a required pointer is NULL");
+    const SampleLayout lay = sample_layout(R * (B + 1), V);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15u))
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_accept_sampled: workspace is NULL or not 16-byte aligned");
+    if (workspace_bytes < lay.total)
+        return fail(DDTREE_ERR_WORKSPACE, "ddtree_accept_sampled: workspace %zu < required %zu bytes", workspace_bytes, lay.total);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = launch_row_argmax(target_logits, dt, row_stride_elems, R, B + 1, V, n_rows, lay.a, workspace, st);
+    if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_accept_sampled: maximum pass: %s", cudaGetErrorString(e));
+    e = launch_row_sample(target_logits, dt, row_stride_elems, R, B + 1, V, n_rows, c, row_uniform, lay, workspace, st);
+    if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_accept_sampled: sampling pass: %s", cudaGetErrorString(e));
+    const int32_t* choice = reinterpret_cast<const int32_t*>(static_cast<const char*>(workspace) + lay.off_tok);
+    e = launch_accept_walk(R, B + 1, L, lay.a, workspace, choice, node_token, node_parent, n_rows, accept_len, accept_nodes,
+                           accept_tokens, bonus_token, node_choice, st);
+    if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_accept_sampled: walk kernel: %s", cudaGetErrorString(e));
     return DDTREE_OK;
 }
 

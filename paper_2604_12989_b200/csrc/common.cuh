@@ -48,10 +48,23 @@ cudaError_t launch_tree_build(int R, int L, int V, int K, int B, const BuildPart
                               float* topk_logprob, cudaStream_t st);
 cudaError_t launch_row_argmax(const void* logits, int dt, int64_t row_stride, int R, int N, int V,
                               const int32_t* n_rows, const ArgmaxLayout& lay, void* ws, cudaStream_t st);
-cudaError_t launch_accept_walk(int R, int N, int L, const ArgmaxLayout& lay, const void* ws,
+// `choice`: NULL = the arg-max of the chunk partials in `ws` is the target's choice at a row; else [R, N] tokens.
+cudaError_t launch_accept_walk(int R, int N, int L, const ArgmaxLayout& lay, const void* ws, const int32_t* choice,
                                const int32_t* node_token, const int32_t* node_parent, const int32_t* n_rows,
                                int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
                                int32_t* bonus_token, int32_t* node_argmax, cudaStream_t st);
+
+// Temperature-based decoding rule: workspace = the arg-max partials, then per (row, chunk) weight sums and the
+// sampled token of every row.
+struct SampleLayout {
+    ArgmaxLayout a;
+    size_t off_sum, off_tok, total;
+};
+SampleLayout sample_layout(int rows, int V);
+// After launch_row_argmax on the same workspace: draws the token of every row into the workspace's token array.
+cudaError_t launch_row_sample(const void* logits, int dt, int64_t row_stride, int R, int N, int V, const int32_t* n_rows,
+                              float log2e_over_t, const uint32_t* row_uniform, const SampleLayout& lay, void* ws,
+                              cudaStream_t st);
 
 struct AttnArgs {
     const void *q, *k_cache, *v_cache, *k_tree, *v_tree;

@@ -4,7 +4,10 @@
 //                          q_i = softmax(l_i), tokens ranked by probability).
 //   row_argmax_kernel   -- per (row, chunk): maximum and the lowest id attaining it (the greedy
 //                          decoding rule of Section 4.4).
-// Both read each element once with 16-byte loads; chunk partials are merged by the kernels in
+//   row_weight_sums_kernel / row_sample_kernel -- the temperature-based decoding rule of Section 4.4:
+//                          per (row, chunk) sums of fixed-point softmax weights, then the inverse-CDF
+//                          draw of every row's token.
+// All read each element once per pass with 16-byte loads; chunk partials are merged by the kernels in
 // tree_build.cu / accept_walk.cu.
 #include "common.cuh"
 #include <math_constants.h>
@@ -186,6 +189,175 @@ row_argmax_kernel(const T* __restrict__ logits, int64_t row_stride, int N, int V
     }
 }
 
+// ---- temperature-based decoding rule ---------------------------------------------------------------
+// The target's choice at a row is a draw from softmax(x / T) (Section 4.4).  The draw is defined on integers so
+// that it does not depend on the order of any sum: token v has the weight
+//     W_v = floor(2^40 * e_v),  e_v = 2^((x_v - max x) * c),  c = float32(log2(e) / T),
+// with e_v evaluated in float32, one rounding per operation: t = (x_v - max) * c; n = t rounded to the nearest
+// integer by adding 1.5 * 2^23 (the integer is then read from the sum's bit pattern); f = t - n in [-1/2, 1/2];
+// a degree-5 polynomial p for 2^f in Horner form, multiply then add; W_v = significand of p shifted by its
+// exponent + n + 17; tokens with t < -40 weigh nothing.  The row's random input k (32 bits) selects the
+// smallest v whose inclusive prefix sum exceeds floor(total * k / 2^32).  No instruction of the weight goes
+// through the conversion unit (16 results per clock and SM): rounding and the float -> fixed-point step are
+// integer operations on bit patterns.
+__device__ __forceinline__ unsigned long long sample_weight(float x, float m, float c) {
+    const float t = __fmul_rn(__fsub_rn(x, m), c);
+    if (!(t >= -40.f)) return 0ull;  // also -inf and NaN
+    const float r = __fadd_rn(t, 12582912.f);
+    const int n = static_cast<int>(__float_as_uint(r)) - 0x4B400000;
+    const float f = __fsub_rn(t, __fsub_rn(r, 12582912.f));
+    float acc = 0.00132647273f;
+    acc = __fadd_rn(__fmul_rn(acc, f), 0.00967151299f);
+    acc = __fadd_rn(__fmul_rn(acc, f), 0.0555073358f);
+    acc = __fadd_rn(__fmul_rn(acc, f), 0.240222424f);
+    acc = __fadd_rn(__fmul_rn(acc, f), 0.693147004f);
+    acc = __fadd_rn(__fmul_rn(acc, f), 1.0f);
+    const unsigned bits = __float_as_uint(acc);
+    const unsigned sig = (bits & 0x7FFFFFu) | 0x800000u;            // p = sig * 2^(e - 23), e in {-1, 0}
+    const int sh = static_cast<int>(bits >> 23) - 127 + 17 + n;     // floor(p * 2^n * 2^40) = sig * 2^(e - 23 + n + 40)
+    return sh >= 0 ? static_cast<unsigned long long>(sig) << sh : static_cast<unsigned long long>(sig >> -sh);
+}
+
+// w[0] + ... + w[e]
+template <int VN>
+__device__ __forceinline__ unsigned long long prefix_to(const unsigned long long (&w)[VN], int e) {
+    unsigned long long s = 0;
+#pragma unroll
+    for (int i = 0; i < VN; ++i)
+        if (i <= e) s += w[i];
+    return s;
+}
+
+// Row maximum from the arg-max pass's chunk partials (every thread reads them all: there are few).
+__device__ __forceinline__ float row_max_of(const float* __restrict__ pval, int chunks) {
+    float m = -CUDART_INF_F;
+    for (int c = 0; c < chunks; ++c) m = fmaxf(m, pval[c]);
+    return m;
+}
+
+__device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v, unsigned long long* sm) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) sm[warp] = v;
+    __syncthreads();
+    unsigned long long t = 0;
+    for (int w = 0; w < kWarps; ++w) t += sm[w];
+    return t;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+row_weight_sums_kernel(const T* __restrict__ logits, int64_t row_stride, int N, int V, const int32_t* __restrict__ n_rows,
+                       int chunk_elems, int chunks, float c, const float* __restrict__ pval,
+                       unsigned long long* __restrict__ psum) {
+    constexpr int VN = Vec16<T>::N;
+    pdl_wait();
+    const int row = blockIdx.x / chunks, chunk = blockIdx.x % chunks;
+    if (row % N >= n_rows[row / N]) return;  // padding row: never read
+    const int tid = threadIdx.x;
+    const float m = row_max_of(pval + static_cast<size_t>(row) * chunks, chunks);
+    const T* x = logits + static_cast<int64_t>(row) * row_stride;
+    const int begin = chunk * chunk_elems;
+    const int end = min(V, begin + chunk_elems);
+    const int vec_end = begin + ((end - begin) / VN) * VN;
+    unsigned long long acc = 0;
+    constexpr int kStep = kThreads * VN;
+    for (int it = begin + tid * VN; it < vec_end; it += kUnroll * kStep) {
+        float vals[kUnroll][VN];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int id0 = it + u * kStep;
+            if (id0 < vec_end) Vec16<T>::load(x + id0, vals[u]);
+            else {
+#pragma unroll
+                for (int e = 0; e < VN; ++e) vals[u][e] = -CUDART_INF_F;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+#pragma unroll
+            for (int e = 0; e < VN; ++e) acc += sample_weight(vals[u][e], m, c);
+    }
+    if (tid < end - vec_end) acc += sample_weight(Vec16<T>::scalar(x + vec_end + tid), m, c);
+    __shared__ unsigned long long sm[kWarps];
+    const unsigned long long total = block_sum_u64(acc, sm);
+    if (tid == 0) psum[static_cast<size_t>(row) * chunks + chunk] = total;
+}
+
+// One CTA per row: find the chunk the threshold falls into from the chunk sums, then the token inside that chunk.
+// The chunk is walked in rounds of 256 x (elements per 16-byte vector) consecutive tokens: every thread weighs
+// its vector, a block scan of the thread sums tells whether the threshold falls into this round and into which
+// thread's vector; otherwise the round's total is taken off the threshold.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+row_sample_kernel(const T* __restrict__ logits, int64_t row_stride, int N, int V, const int32_t* __restrict__ n_rows,
+                  int chunk_elems, int chunks, float c, const float* __restrict__ pval,
+                  const unsigned long long* __restrict__ psum, const uint32_t* __restrict__ row_uniform,
+                  int32_t* __restrict__ token) {
+    constexpr int VN = Vec16<T>::N;
+    pdl_wait();
+    const int row = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (row % N >= n_rows[row / N]) {
+        if (tid == 0) token[row] = -1;
+        return;
+    }
+    const float m = row_max_of(pval + static_cast<size_t>(row) * chunks, chunks);
+    const unsigned long long* ps = psum + static_cast<size_t>(row) * chunks;
+    unsigned long long total = 0;
+    for (int k = 0; k < chunks; ++k) total += ps[k];
+    if (total == 0) {  // no finite maximum in the row: nothing to draw from
+        if (tid == 0) token[row] = -1;
+        return;
+    }
+    const unsigned long long u = row_uniform[row];
+    unsigned long long thr = (__umul64hi(total, u) << 32) | ((total * u) >> 32);  // floor(total * u / 2^32) < total
+    int chunk = 0;
+    while (chunk + 1 < chunks && thr >= ps[chunk]) thr -= ps[chunk++];  // thr is now relative to the chunk's first token
+    const T* x = logits + static_cast<int64_t>(row) * row_stride;
+    const int end = min(V, (chunk + 1) * chunk_elems);
+    __shared__ unsigned long long warp_total[kWarps];
+    for (int base = chunk * chunk_elems; base < end; base += kThreads * VN) {  // chunk starts are multiples of 2048
+        const int id0 = base + tid * VN;
+        float vals[VN];
+        if (id0 + VN <= end) {
+            Vec16<T>::load(x + id0, vals);
+        } else {
+#pragma unroll
+            for (int e = 0; e < VN; ++e) vals[e] = id0 + e < end ? Vec16<T>::scalar(x + id0 + e) : -CUDART_INF_F;
+        }
+        unsigned long long w[VN], mine = 0;
+#pragma unroll
+        for (int e = 0; e < VN; ++e) { w[e] = sample_weight(vals[e], m, c); mine += w[e]; }
+        unsigned long long incl = mine;  // inclusive scan over the warp, then over the warps
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long up = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) warp_total[warp] = incl;
+        __syncthreads();
+        unsigned long long round_total = 0;
+        for (int k = 0; k < kWarps; ++k) {
+            if (k < warp) incl += warp_total[k];
+            round_total += warp_total[k];
+        }
+        if (thr < round_total) {  // the same for every thread
+            unsigned long long acc = incl - mine;
+            if (acc <= thr && thr < incl) {  // exactly one thread: the inclusive sums never decrease
+                int found = id0 + VN - 1;
+#pragma unroll
+                for (int e = VN - 1; e >= 0; --e)
+                    if (acc + prefix_to<VN>(w, e) > thr) found = id0 + e;
+                token[row] = found;
+            }
+            return;
+        }
+        thr -= round_total;
+        __syncthreads();  // warp_total is rewritten in the next round
+    }
+}
+
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 int pick_chunk(int64_t rows, int V, int lo, int hi) {
@@ -254,6 +426,41 @@ cudaError_t launch_row_argmax(const void* logits, int dt, int64_t row_stride, in
     return launch_pdl(row_argmax_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), 0, st,
                       static_cast<const __nv_bfloat16*>(logits), row_stride, N, V, n_rows, lay.chunk_elems, lay.chunks,
                       pval, pid);
+}
+
+SampleLayout sample_layout(int rows, int V) {
+    SampleLayout lay;
+    lay.a = argmax_layout(rows, V);
+    lay.off_sum = lay.a.total;
+    lay.off_tok = align_up(lay.off_sum + static_cast<size_t>(rows) * lay.a.chunks * 8, 256);
+    lay.total = align_up(lay.off_tok + static_cast<size_t>(rows) * 4, 256);
+    return lay;
+}
+
+cudaError_t launch_row_sample(const void* logits, int dt, int64_t row_stride, int R, int N, int V, const int32_t* n_rows,
+                              float log2e_over_t, const uint32_t* row_uniform, const SampleLayout& lay, void* ws,
+                              cudaStream_t st) {
+    char* w = static_cast<char*>(ws);
+    const float* pval = reinterpret_cast<const float*>(w + lay.a.off_val);
+    unsigned long long* psum = reinterpret_cast<unsigned long long*>(w + lay.off_sum);
+    int32_t* token = reinterpret_cast<int32_t*>(w + lay.off_tok);
+    const unsigned rows = static_cast<unsigned>(R) * N;
+    const unsigned grid = static_cast<unsigned>(lay.a.chunks) * rows;
+    cudaError_t e;
+    if (dt == DDTREE_F32) {
+        e = launch_pdl(row_weight_sums_kernel<float>, dim3(grid), dim3(kThreads), 0, st, static_cast<const float*>(logits),
+                       row_stride, N, V, n_rows, lay.a.chunk_elems, lay.a.chunks, log2e_over_t, pval, psum);
+        if (e != cudaSuccess) return e;
+        return launch_pdl(row_sample_kernel<float>, dim3(rows), dim3(kThreads), 0, st, static_cast<const float*>(logits),
+                          row_stride, N, V, n_rows, lay.a.chunk_elems, lay.a.chunks, log2e_over_t, pval, psum, row_uniform, token);
+    }
+    e = launch_pdl(row_weight_sums_kernel<__nv_bfloat16>, dim3(grid), dim3(kThreads), 0, st,
+                   static_cast<const __nv_bfloat16*>(logits), row_stride, N, V, n_rows, lay.a.chunk_elems, lay.a.chunks,
+                   log2e_over_t, pval, psum);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(row_sample_kernel<__nv_bfloat16>, dim3(rows), dim3(kThreads), 0, st,
+                      static_cast<const __nv_bfloat16*>(logits), row_stride, N, V, n_rows, lay.a.chunk_elems, lay.a.chunks,
+                      log2e_over_t, pval, psum, row_uniform, token);
 }
 
 }  // namespace ddtree

@@ -65,3 +65,13 @@ def test_validation_without_gpu(lib):
     assert lib.ddtree_kv_compact(1, 8, 4, 2, 64, 1, 2, ptrs, bad, ptrs, ptrs, p, p, p, None) == 1        # misaligned layer buffer
     assert lib.ddtree_kv_compact(1, 8, 4, 2, 64, 9, 2, ptrs, ptrs, ptrs, ptrs, p, p, p, None) == 1       # bad dtype
     assert lib.ddtree_kv_compact(1, 8, 4, 2, 64, 1, 0, ptrs, ptrs, ptrs, ptrs, p, p, p, None) == 1       # no layers
+    # ddtree_accept_sampled: temperature and pointers are checked on the host
+    sampled = lambda T, u=p: lib.ddtree_accept_sampled(p, 0, 8, 1, 1, 8, 1, p, p, p, T, u, p, p, p, p, None, p, 1 << 20, None)
+    assert sampled(0.0) == 1 and b"temperature" in lib.ddtree_last_error()
+    assert sampled(-2.0) == 1
+    assert sampled(float("inf")) == 1
+    assert sampled(float("nan")) == 1
+    assert sampled(1.0, None) == 1 and b"NULL" in lib.ddtree_last_error()                                # no random inputs
+    assert lib.ddtree_accept_sampled(p, 0, 8, 1, 1, 8, 1, p, p, p, 1.0, p, p, p, p, p, None, p, 16, None) == 3  # workspace too small
+    assert lib.ddtree_accept_sampled_workspace_bytes(1, 64, 151936) > lib.ddtree_accept_workspace_bytes(1, 64, 151936)
+    assert lib.ddtree_accept_sampled_workspace_bytes(1, 4096, 151936) == 0                               # B out of range
