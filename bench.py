@@ -256,20 +256,33 @@ def run_gpu(args, w):
     target = up(target_h, bf)
 
     ws_build = torch.empty(max(256, dd.lib().ddtree_build_workspace_bytes(w.R, w.L, w.V, w.K, w.B)), dtype=torch.uint8, device=dev)
-    ws_acc = torch.empty(max(256, dd.lib().ddtree_accept_workspace_bytes(w.R, w.B, w.V)), dtype=torch.uint8, device=dev)
+    T = float(args.temperature)
+    ws_acc = torch.empty(max(256, (dd.lib().ddtree_accept_sampled_workspace_bytes if T > 0 else
+                                   dd.lib().ddtree_accept_workspace_bytes)(w.R, w.B, w.V)), dtype=torch.uint8, device=dev)
+    # temperature > 0: one 32-bit random input per row, drawn once with a seeded generator (they are inputs of the
+    # call; a serving loop would refresh them on the device every round)
+    row_uniform = torch.from_numpy(np.random.default_rng(seed + 17).integers(0, 2 ** 32, (w.R, w.N), dtype=np.uint64)
+                                   .astype(np.uint32).view(np.int32)).to(dev)
+
+    def accept_call(tgt, out=None):
+        if T > 0:
+            return dd.ddtree_accept_sampled(tgt, w.L, tree.node_token, tree.node_parent, tree.n_rows, T, row_uniform,
+                                            workspace=ws_acc, out=out)
+        return dd.ddtree_accept(tgt, w.L, tree.node_token, tree.node_parent, tree.n_rows, workspace=ws_acc, out=out)
+
     ws_att = torch.empty(max(256, dd.tree_attention_workspace_bytes(w.R, w.B, w.Hq, w.Hkv, w.d, 1 if bf else 0, cu_host)),
                          dtype=torch.uint8, device=dev)
-    acc = dd.ddtree_accept(target, w.L, tree.node_token, tree.node_parent, tree.n_rows, workspace=ws_acc)
+    acc = accept_call(target)
 
     def one_round(layer_inputs=layers, tgt=target, lg=logits):
         dd.ddtree_build(lg, w.K, w.B, roots, plen, workspace=ws_build, out=tree)
         for l, (q, kc, vc, kt, vt) in enumerate(layer_inputs):
             dd.ddtree_tree_attention(q, kc, vc, cu_host, cu, kt, vt, tree.anc_mask, tree.n_rows, out=outs[l & 1],
                                      workspace=ws_att)
-        dd.ddtree_accept(tgt, w.L, tree.node_token, tree.node_parent, tree.n_rows, workspace=ws_acc, out=acc)
+        accept_call(tgt, acc)
 
     attn_kernels = 2 if (bf and ws_att.numel() > 256) else 1  # split-KV adds the combine kernel
-    launches_per_round = 2 + attn_kernels * w.layers + 2
+    launches_per_round = 2 + attn_kernels * w.layers + (4 if T > 0 else 2)
 
     # ---- capture one round in a CUDA graph (launch-bound otherwise: ~40 host calls per round) ----
     stream = torch.cuda.Stream(device=dev)
@@ -346,8 +359,7 @@ def run_gpu(args, w):
     att_call_ms = ga.elapsed_time(gb) / ((reps - 3) * w.layers)
     stage_ms = {}
     for name, fn in (("build", lambda: dd.ddtree_build(logits, w.K, w.B, roots, plen, workspace=ws_build, out=tree)),
-                     ("accept", lambda: dd.ddtree_accept(target, w.L, tree.node_token, tree.node_parent, tree.n_rows,
-                                                         workspace=ws_acc, out=acc))):
+                     ("accept", lambda: accept_call(target, acc))):
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
         ts = []
         for it in range(8):
@@ -471,6 +483,7 @@ def run_gpu(args, w):
                    "layers": w.layers, "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2: every layer has its own K/V cache (%.0f MB per round)" %
                          ((byt * w.layers + w.R * w.L * w.V * 4 + w.R * w.N * w.V * 2) / 1e6),
+                   "decoding": "greedy" if T <= 0 else f"temperature {T:g} (ddtree_accept_sampled)",
                    "launch": "one round captured in a CUDA graph and replayed"},
         "tokens_per_s": float((accept_len + 1).sum()) * world / (ms_per_step * 1e-3),
         "accept_len_mean": float(accept_len.mean()),
@@ -500,6 +513,9 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="workload index (1 = the Qwen3-8B-shaped single request)")
     ap.add_argument("--variant", default="lit", choices=wl.VARIANTS)
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling small cases only)")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="0 = the greedy decoding rule (the benchmark's metric); > 0: the verifier walk samples the target's "
+                         "choice at that temperature (ddtree_accept_sampled)")
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     args = ap.parse_args()
     w = wl.WORKLOADS[args.config]

@@ -214,8 +214,9 @@ __device__ __forceinline__ unsigned long long sample_weight(float x, float m, fl
     acc = __fadd_rn(__fmul_rn(acc, f), 1.0f);
     const unsigned bits = __float_as_uint(acc);
     const unsigned sig = (bits & 0x7FFFFFu) | 0x800000u;            // p = sig * 2^(e - 23), e in {-1, 0}
-    const int sh = static_cast<int>(bits >> 23) - 127 + 17 + n;     // floor(p * 2^n * 2^40) = sig * 2^(e - 23 + n + 40)
-    return sh >= 0 ? static_cast<unsigned long long>(sig) << sh : static_cast<unsigned long long>(sig >> -sh);
+    // floor(p * 2^n * 2^40) = floor(sig * 2^(e + 17 + n)): a constant left shift, then a right shift by -(e + n) in [0, 41]
+    const int down = 127 - static_cast<int>(bits >> 23) - n;
+    return (static_cast<unsigned long long>(sig) << 17) >> down;
 }
 
 // w[0] + ... + w[e]
