@@ -129,3 +129,20 @@ def test_argument_errors():
         assert e.value.status == 1
     with pytest.raises(dd.DDTreeError):
         dd.ddtree_accept_sampled(t, w.L, tok, par, n_rows, 1.0, u, workspace=torch.empty(256, dtype=torch.uint8).cuda())
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_shapes(seed):
+    rng = np.random.default_rng(100 + seed)
+    R = int(rng.integers(1, 5))
+    B = int(rng.choice([1, 2, 7, 16, 33, 64]))
+    V = int(rng.choice([9, 64, 257, 4099, 8192, 8193, 16385]))
+    K = int(min(V, rng.integers(1, 5)))
+    dtype = str(rng.choice(["f32", "bf16"]))
+    T = float(rng.choice([0.25, 0.9, 1.0, 3.0]))
+    w = wl.small_workload(R=R, L=int(rng.integers(2, 9)), V=V, K=K, B=B, Hq=4, Hkv=2, d=64, dtype=dtype,
+                          prefix_lens=tuple(int(x) for x in rng.integers(0, 20, R)), index=80 + seed)
+    trees = make_trees(w)
+    tl = np.stack([wl.target_logits(w, trees[r].depth, r, "peak") for r in range(w.R)])
+    ks = rng.integers(0, 2 ** 32, (w.R, w.N), dtype=np.uint64)
+    run_and_compare(w, trees, tl, T, ks)
