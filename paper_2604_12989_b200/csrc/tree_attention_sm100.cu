@@ -495,7 +495,7 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
             // ~850 cycles; the barriers are tested together beforehand to keep it from draining.
             const int s = j % kTailVStages, g = j & 1, b = (j >> 1) & 1;  // key group and its P^T buffer
             const bool more = j + kTailSBufs < my_tiles;
-            const bool st8 = j == kStampTile;
+            [[maybe_unused]] const bool st8 = j == kStampTile;
             STAMP(st8, 0);
             const bool k_ok = !more || mbar_test(smem_u32(&sm.k_full[(j + kTailSBufs) % kTailKStages]), ((j + kTailSBufs) / kTailKStages) & 1);
             const bool ready = mbar_test(smem_u32(&sm.v_full[s]), (j / kTailVStages) & 1) & k_ok &
@@ -560,7 +560,7 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
         STAMP_DECL;
         for (int q = 0; q < my_count; ++q) {
             const int j = 2 * q + g, t = t_begin + j, b = q & 1, sb = j % kTailSBufs;
-            const bool st8 = j == kStampTile;
+            [[maybe_unused]] const bool st8 = j == kStampTile;
             STAMP(st8, 0);
             STAMP(j == kStampTile + 2, 8);
             STAMP(j == kStampTile + 8, 9);
@@ -892,7 +892,7 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         }
         STAMP_DECL;
         for (int j = 0; j < my_tiles && ok; ++j) {
-            const bool st8 = j == kStampTile, st9 = j == kStampTile + 1;
+            [[maybe_unused]] const bool st8 = j == kStampTile, st9 = j == kStampTile + 1;
             STAMP(st8 || st9, st8 ? 0 : 3);
             // One burst per tile: O_h += P_h V_h for both column halves of tile j, then the scores of
             // tile j+2 into the S buffer those P halves sat in.  The tensor pipe pays a start-up
@@ -1015,7 +1015,7 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         for (int j = 1; j < my_tiles && ok; ++j) {
             const int t = t_begin + j, b = j % kSBufs;
             const uint32_t s_addr = lane_addr + kColS + b * kTile + half * 64;
-            const bool st8 = j == kStampTile;
+            [[maybe_unused]] const bool st8 = j == kStampTile;
             STAMP(st8, 0);
             STAMP(j == kStampTile + 1, 8);
             STAMP(j == kStampTile + 2, 9);
