@@ -353,6 +353,26 @@ def node_sampled(target_logits: np.ndarray, temperature: float, uniforms: np.nda
                      for i in range(target_logits.shape[0])], np.int32)
 
 
+# --------------------------------------------------------------------------
+# Section 4.4: position ids by tree depth, consumed by the verifier's positional encoding
+# --------------------------------------------------------------------------
+
+
+def rope(x: np.ndarray, positions: np.ndarray, theta: float) -> np.ndarray:
+    """Rotary positional encoding of the rows of x ([rows, heads, d], d even) at the given integer
+    positions ("we assign position ids by tree depth so that the verifier applies the correct positional
+    encoding", Section 4.4; the target models of the paper, Qwen3, use rotary embeddings in the
+    half-split form).  Pair (j, j + d/2) of every head is rotated by the angle
+    positions[row] * theta^(-2j/d): as complex numbers z_j = x_j + i x_{j+d/2}, out = z_j * exp(i * angle)."""
+    x = np.asarray(x, np.float64)
+    rows, heads, d = x.shape
+    half = d // 2
+    inv_freq = float(theta) ** (-np.arange(half, dtype=np.float64) * 2.0 / d)
+    ang = np.asarray(positions, np.float64)[:, None] * inv_freq[None, :]
+    z = (x[..., :half] + 1j * x[..., half:]) * np.exp(1j * ang)[:, None, :]
+    return np.concatenate([z.real, z.imag], axis=-1)
+
+
 def kv_compact(cache: np.ndarray, tree_rows: np.ndarray, prefix_len: int, path: Sequence[int]) -> np.ndarray:
     """End of a round (Section 4.4: after the walk only the accepted path stays in
     the cache): the keys (or values) of the root and of the accepted nodes are

@@ -610,3 +610,31 @@ def test_sampled_walk_reduces_to_the_greedy_walk_at_low_temperature():
     cold = orc.accept_walk(tree.token, tree.parent, tree.n_rows, orc.node_sampled(target, 1e-3, ks))
     assert (cold.accept_len, cold.nodes, cold.bonus_token) == (greedy.accept_len, greedy.nodes, greedy.bonus_token)
     assert greedy.accept_len >= 1
+
+
+# --------------------------------------------------------------------------
+# Rotary positional encoding at the tree's position ids
+# --------------------------------------------------------------------------
+
+def test_rope_against_the_real_valued_textbook_form():
+    rng = np.random.default_rng(20)
+    x = rng.standard_normal((5, 3, 8))
+    pos = np.array([0, 1, 7, 100, 4097])
+    out = orc.rope(x, pos, 10000.0)
+    for r in range(5):
+        for j in range(4):
+            a = pos[r] * 10000.0 ** (-2.0 * j / 8)
+            c, s = math.cos(a), math.sin(a)
+            np.testing.assert_allclose(out[r, :, j], x[r, :, j] * c - x[r, :, j + 4] * s, atol=1e-12)
+            np.testing.assert_allclose(out[r, :, j + 4], x[r, :, j + 4] * c + x[r, :, j] * s, atol=1e-12)
+    np.testing.assert_array_equal(out[0], x[0])                     # position 0 is the identity
+
+
+def test_rope_preserves_norms_and_makes_scores_depend_on_the_distance_only():
+    rng = np.random.default_rng(21)
+    q, k = rng.standard_normal((1, 1, 64)), rng.standard_normal((1, 1, 64))
+    np.testing.assert_allclose(np.linalg.norm(orc.rope(q, [12345], 1e6)), np.linalg.norm(q), rtol=1e-12)
+    dots = [float(np.sum(orc.rope(q, [m], 1e6) * orc.rope(k, [m - 9], 1e6))) for m in (9, 50, 4000)]
+    np.testing.assert_allclose(dots, dots[0], rtol=1e-9)            # <R_m q, R_n k> is a function of m - n
+    # composition: rotating by m and then by n is rotating by m + n
+    np.testing.assert_allclose(orc.rope(orc.rope(q, [30], 1e6), [12], 1e6), orc.rope(q, [42], 1e6), atol=1e-12)
