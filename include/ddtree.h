@@ -207,6 +207,25 @@ int ddtree_accept_sampled(const void* target_logits, int dt, int64_t row_stride_
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * ddtree_rope_tree -- Section 4.4: "we assign position ids by tree depth so that the verifier applies the
+ * correct positional encoding".  Applies the rotary positional encoding (half-split form, as the paper's
+ * Qwen3 targets use) to the tree's query and key rows IN PLACE, at the position ids ddtree_build wrote:
+ * for every valid row i, every head and every j < d/2, with a = position_ids[r, i] * rope_theta^(-2j/d),
+ *     (x[j], x[j + d/2])  <-  (x[j] cos a - x[j + d/2] sin a,  x[j + d/2] cos a + x[j] sin a).
+ * Angles are evaluated in double precision, the rotation in float32, results rounded to dt.
+ * Call it on a layer's q and k_tree before ddtree_tree_attention (the cached keys were rotated when they
+ * were produced).  A pass of its own rather than a step inside the attention kernel: there every K row would
+ * be rotated again by each CTA that loads it.
+ *
+ *   q        [R, B+1, Hq, d]  or NULL      k_tree  [R, B+1, Hkv, d]  or NULL   (not both NULL), dt = F32 or BF16
+ *   position_ids [R, B+1], n_rows [R]      as written by ddtree_build; rows >= n_rows[r] are left untouched
+ *   d even, 2..256; rope_theta > 0 (10^6 for Qwen3)
+ * Errors: DDTREE_ERR_INVALID_ARG / DDTREE_ERR_UNSUPPORTED before anything is launched.
+ * ------------------------------------------------------------------------------------------ */
+int ddtree_rope_tree(void* q, void* k_tree, const int32_t* position_ids, const int32_t* n_rows,
+                     int dt, int R, int B, int Hq, int Hkv, int d, float rope_theta, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * ddtree_accept_static_scratch -- the paper has no counterpart; this is a packaging variant of
  * ddtree_accept for callers that cannot hand over a workspace.
  *

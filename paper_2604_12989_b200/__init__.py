@@ -23,7 +23,7 @@ EXPORTS = (
     "ddtree_tree_attention_workspace_bytes", "ddtree_tree_attention",
     "ddtree_accept_workspace_bytes", "ddtree_accept", "ddtree_accept_static_scratch",
     "ddtree_accept_sampled_workspace_bytes", "ddtree_accept_sampled",
-    "ddtree_kv_compact",
+    "ddtree_kv_compact", "ddtree_rope_tree",
     "ddtree_device_status",
 )
 
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.ddtree_accept_sampled_workspace_bytes.argtypes = [i32] * 3
         L.ddtree_accept_sampled.restype = i32
         L.ddtree_accept_sampled.argtypes = [vp, i32, i64, i32, i32, i32, i32] + [vp] * 3 + [f32, vp] + [vp] * 5 + [vp, sz, vp]
+        L.ddtree_rope_tree.restype = i32
+        L.ddtree_rope_tree.argtypes = [vp, vp, vp, vp] + [i32] * 6 + [f32, vp]
         L.ddtree_kv_compact.restype = i32
         L.ddtree_kv_compact.argtypes = [i32] * 7 + [vp] * 7 + [vp]
         L.ddtree_device_status.restype = i32
@@ -251,6 +253,20 @@ def ddtree_accept_static_scratch(target_logits, L: int, node_token, node_parent,
         out.accept_nodes.data_ptr(), out.accept_tokens.data_ptr(), out.bonus_token.data_ptr(),
         _ptr(out.node_argmax), _stream(stream)))
     return out
+
+
+def ddtree_rope_tree(q, k_tree, position_ids, n_rows, rope_theta: float, stream=None) -> None:
+    """Rotary positional encoding, in place, of the tree's query rows q [R, B+1, Hq, d] and key rows k_tree
+    [R, B+1, Hkv, d] (either may be None) at the position ids written by ddtree_build."""
+    t = q if q is not None else k_tree
+    assert t is not None and t.is_cuda and t.is_contiguous()
+    R, N, _, d = t.shape
+    Hq = q.shape[2] if q is not None else 1
+    Hkv = k_tree.shape[2] if k_tree is not None else 1
+    for u in (q, k_tree):
+        assert u is None or (u.is_cuda and u.is_contiguous() and u.dtype == t.dtype and u.shape[0] == R and u.shape[1] == N and u.shape[3] == d)
+    _check(lib().ddtree_rope_tree(_ptr(q), _ptr(k_tree), position_ids.data_ptr(), n_rows.data_ptr(), _dtype_code(t),
+                                  R, N - 1, Hq, Hkv, d, float(rope_theta), _stream(stream)))
 
 
 def ddtree_kv_compact(k_tree, v_tree, k_cache, v_cache, dst_row, accept_len, accept_nodes, stream=None) -> None:

@@ -170,6 +170,22 @@ int ddtree_accept_sampled(const void* target_logits, int dt, int64_t row_stride_
     return DDTREE_OK;
 }
 
+int ddtree_rope_tree(void* q, void* k_tree, const int32_t* position_ids, const int32_t* n_rows, int dt, int R, int B,
+                     int Hq, int Hkv, int d, float rope_theta, void* cuda_stream) {
+    if (R < 1 || B < 1 || Hq < 1 || Hkv < 1) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_rope_tree: R, B, Hq, Hkv must be >= 1");
+    if (B > kMaxB) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_rope_tree: B %d > %d", B, kMaxB);
+    if (dt != DDTREE_F32 && dt != DDTREE_BF16) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_rope_tree: unknown dtype %d", dt);
+    if (d < 2 || d > 256 || (d & 1)) return fail(DDTREE_ERR_UNSUPPORTED, "ddtree_rope_tree: head_dim %d must be even and in [2, 256]", d);
+    if (!(rope_theta > 0.f) || !(rope_theta <= 3.0e38f))
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_rope_tree: rope_theta must be positive and finite");
+    if (!position_ids || !n_rows) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_rope_tree: position_ids or n_rows is NULL");
+    if (!q && !k_tree) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_rope_tree: both q and k_tree are NULL");
+    const cudaError_t e = launch_rope_tree(q, k_tree, position_ids, n_rows, dt, R, B + 1, Hq, Hkv, d,
+                                           std::log2(static_cast<double>(rope_theta)), static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_rope_tree: %s", cudaGetErrorString(e));
+    return DDTREE_OK;
+}
+
 int ddtree_kv_compact(int R, int B, int L, int Hkv, int d, int dt, int layers, const void* const* k_tree,
                       const void* const* v_tree, void* const* k_cache, void* const* v_cache, const int64_t* dst_row,
                       const int32_t* accept_len, const int32_t* accept_nodes, void* cuda_stream) {

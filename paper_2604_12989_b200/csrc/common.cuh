@@ -66,6 +66,10 @@ cudaError_t launch_row_sample(const void* logits, int dt, int64_t row_stride, in
                               float log2e_over_t, const uint32_t* row_uniform, const SampleLayout& lay, void* ws,
                               cudaStream_t st);
 
+// Rotary positional encoding of the tree's Q / K rows, in place (either pointer may be NULL).
+cudaError_t launch_rope_tree(void* q, void* k, const int32_t* position_ids, const int32_t* n_rows, int dt, int R, int N,
+                             int Hq, int Hkv, int d, double log2_theta, cudaStream_t st);
+
 struct AttnArgs {
     const void *q, *k_cache, *v_cache, *k_tree, *v_tree;
     const int32_t* cu_prefix;

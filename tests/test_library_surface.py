@@ -75,3 +75,11 @@ def test_validation_without_gpu(lib):
     assert lib.ddtree_accept_sampled(p, 0, 8, 1, 1, 8, 1, p, p, p, 1.0, p, p, p, p, p, None, p, 16, None) == 3  # workspace too small
     assert lib.ddtree_accept_sampled_workspace_bytes(1, 64, 151936) > lib.ddtree_accept_workspace_bytes(1, 64, 151936)
     assert lib.ddtree_accept_sampled_workspace_bytes(1, 4096, 151936) == 0                               # B out of range
+    # ddtree_rope_tree
+    rope = lambda d=128, theta=1e6, q=p, k=p, dt=1: lib.ddtree_rope_tree(q, k, p, p, dt, 1, 8, 4, 2, d, theta, None)
+    assert rope(d=7) == 2 and b"head_dim" in lib.ddtree_last_error()      # odd head dimension
+    assert rope(d=512) == 2
+    assert rope(theta=0.0) == 1 and rope(theta=float("inf")) == 1
+    assert rope(q=None, k=None) == 1
+    assert rope(dt=5) == 1
+    assert lib.ddtree_rope_tree(p, p, None, p, 1, 1, 8, 4, 2, 128, 1e6, None) == 1   # no position ids
