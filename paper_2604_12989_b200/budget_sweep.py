@@ -9,7 +9,8 @@ the tree is built, target logits for its nodes are drawn on the device (noise pl
 true token per depth; the drafter's boost is about as large as the largest of the V noise draws and
 shrinks with depth, so the true token is often not the drafter's first choice and a larger tree catches
 more of it; the target always prefers the true token); then, timed with CUDA events,
-ddtree_build -> one ddtree_tree_attention per layer -> ddtree_accept -> ddtree_kv_compact, after which
+ddtree_build -> one ddtree_tree_attention per layer (after ddtree_rope_tree with --rope-theta) -> ddtree_accept
+(ddtree_accept_sampled with --temperature) -> ddtree_kv_compact, after which
 the accepted path is part of the KV cache and the prefix has grown by accept_len + 1.  There is no
 model behind the logits, so the acceptance lengths are those of the recipe, not of Qwen3; what the
 sweep shows on this GPU is how the cost of a round grows with the budget and where tokens/s peaks
@@ -23,7 +24,7 @@ import statistics
 import numpy as np
 
 
-def run(budgets, rounds, layers, prefix, seed=0, draft_boost0=4.9, draft_slope=0.1):
+def run(budgets, rounds, layers, prefix, seed=0, draft_boost0=4.9, draft_slope=0.1, temperature=0.0, rope_theta=0.0):
     import torch
     import paper_2604_12989_b200 as dd
     from paper_2604_12989_b200 import workloads as wl
@@ -49,7 +50,7 @@ def run(budgets, rounds, layers, prefix, seed=0, draft_boost0=4.9, draft_slope=0
         boost = torch.from_numpy(wl._boost(w, 0, depth_tab, "peak", seed)).to(dev)           # target: boost of depth 1..L+1
         draft_boost = torch.from_numpy(((draft_boost0 - draft_slope * depth_tab) * w.noise).astype(np.float32)).to(dev)
         ws_b = torch.empty(max(256, dd.lib().ddtree_build_workspace_bytes(1, w.L, w.V, K, B)), dtype=torch.uint8, device=dev)
-        ws_a = torch.empty(max(256, dd.lib().ddtree_accept_workspace_bytes(1, B, w.V)), dtype=torch.uint8, device=dev)
+        ws_a = torch.empty(max(256, dd.lib().ddtree_accept_sampled_workspace_bytes(1, B, w.V)), dtype=torch.uint8, device=dev)
         roots = torch.zeros(1, dtype=torch.int32, device=dev)
         P = prefix
         times, lens, rows = [], [], []
@@ -76,9 +77,16 @@ def run(budgets, rounds, layers, prefix, seed=0, draft_boost0=4.9, draft_slope=0
             e0.record()
             dd.ddtree_build(logits, K, B, roots, plen, workspace=ws_b, out=tree)
             for l in range(layers):
+                if rope_theta > 0:  # the tree's Q / K rows of this layer at their position ids (in place: the synthetic
+                    dd.ddtree_rope_tree(qs[l], kt[l], tree.position_ids, tree.n_rows, rope_theta)  # rows are reused as they are)
                 dd.ddtree_tree_attention(qs[l], kc[l][:P], vc[l][:P], cu_host, cu, kt[l], vt[l], tree.anc_mask, tree.n_rows,
                                          out=outs[l & 1], workspace=ws_t)
-            acc = dd.ddtree_accept(target, w.L, tree.node_token, tree.node_parent, tree.n_rows, workspace=ws_a, out=acc)
+            if temperature > 0:
+                uni = torch.randint(-2 ** 31, 2 ** 31 - 1, (1, w.N), generator=gen, device=dev, dtype=torch.int32)
+                acc = dd.ddtree_accept_sampled(target, w.L, tree.node_token, tree.node_parent, tree.n_rows, temperature, uni,
+                                               workspace=ws_a, out=acc)
+            else:
+                acc = dd.ddtree_accept(target, w.L, tree.node_token, tree.node_parent, tree.n_rows, workspace=ws_a, out=acc)
             dd.ddtree_kv_compact(kt, vt, kc, vc, dst, acc.accept_len, acc.accept_nodes)
             e1.record()
             torch.cuda.synchronize()
@@ -106,9 +114,13 @@ def main():
     ap.add_argument("--prefix", type=int, default=4096)
     ap.add_argument("--draft-boost0", type=float, default=4.9, help="drafter boost of the true token at depth 0, in noise sigmas")
     ap.add_argument("--draft-slope", type=float, default=0.1, help="decrease of that boost per depth, in noise sigmas")
+    ap.add_argument("--temperature", type=float, default=0.0, help="> 0: the walk samples the target's choice (ddtree_accept_sampled)")
+    ap.add_argument("--rope-theta", type=float, default=0.0, help="> 0: rotate every layer's tree Q / K rows first (ddtree_rope_tree)")
     a = ap.parse_args()
-    res = run([int(x) for x in a.budgets.split(",")], a.rounds, a.layers, a.prefix, 0, a.draft_boost0, a.draft_slope)
-    print(json.dumps({"sweep": res, "layers": a.layers, "prefix": a.prefix, "rounds": a.rounds, "launch": "eager (host-issued calls)"}))
+    res = run([int(x) for x in a.budgets.split(",")], a.rounds, a.layers, a.prefix, 0, a.draft_boost0, a.draft_slope,
+              a.temperature, a.rope_theta)
+    print(json.dumps({"sweep": res, "layers": a.layers, "prefix": a.prefix, "rounds": a.rounds, "temperature": a.temperature,
+                      "rope_theta": a.rope_theta, "launch": "eager (host-issued calls)"}))
 
 
 if __name__ == "__main__":
