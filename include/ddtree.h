@@ -288,6 +288,16 @@ int ddtree_kv_compact(int R, int B, int L, int Hkv, int d, int dt, int layers,
  * reads and clears the word. */
 int ddtree_device_status(void);
 
+/* Self-test of that reporting path (no counterpart in the paper).  Every wait inside the attention
+ * kernel (on a TMA copy, on the tensor pipe, on another warp) polls a bounded number of times; when
+ * the bound runs out the kernel raises the time-out flag in the status word, waits for its own
+ * copies in flight, frees its tensor memory and returns: the context stays usable and no output is
+ * trusted.  This call enqueues a one-thread kernel with such a wait on a barrier that nothing ever
+ * arrives at and a bound of a few thousand polls (microseconds), so that after it
+ * ddtree_device_status() returns DDTREE_ERR_DEVICE_TIMEOUT once and DDTREE_OK afterwards.  The
+ * kernel does not trap, fault or spin without bound. */
+int ddtree_selftest_wait_timeout(void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

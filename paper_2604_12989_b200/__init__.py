@@ -24,7 +24,7 @@ EXPORTS = (
     "ddtree_accept_workspace_bytes", "ddtree_accept", "ddtree_accept_static_scratch",
     "ddtree_accept_sampled_workspace_bytes", "ddtree_accept_sampled",
     "ddtree_kv_compact", "ddtree_rope_tree",
-    "ddtree_device_status",
+    "ddtree_device_status", "ddtree_selftest_wait_timeout",
 )
 
 _lib = None
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.ddtree_kv_compact.argtypes = [i32] * 7 + [vp] * 7 + [vp]
         L.ddtree_device_status.restype = i32
         L.ddtree_device_status.argtypes = []
+        L.ddtree_selftest_wait_timeout.restype = i32
+        L.ddtree_selftest_wait_timeout.argtypes = [vp]
         _lib = L
     return _lib
 
@@ -289,6 +291,12 @@ def ddtree_kv_compact(k_tree, v_tree, k_cache, v_cache, dst_row, accept_len, acc
     _check(lib().ddtree_kv_compact(R, N - 1, L, Hkv, d, _dtype_code(k_tree[0]), layers, arr(k_tree), arr(v_tree),
                                    arr(k_cache), arr(v_cache), dst_row.data_ptr(), accept_len.data_ptr(),
                                    accept_nodes.data_ptr(), _stream(stream)))
+
+
+def selftest_wait_timeout(stream=None) -> None:
+    """Enqueue the library's one-thread kernel whose bounded wait runs out (see include/ddtree.h); the next
+    device_status() raises DDTreeError with status 5 (device-side wait timed out), the one after passes."""
+    _check(lib().ddtree_selftest_wait_timeout(_stream(stream)))
 
 
 def device_status() -> None:

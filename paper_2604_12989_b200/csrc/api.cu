@@ -331,6 +331,12 @@ int ddtree_accept_static_scratch(const void* target_logits, int dt, int64_t row_
                          cuda_stream);
 }
 
+int ddtree_selftest_wait_timeout(void* cuda_stream) {
+    const cudaError_t e = launch_wait_timeout_selftest(4096u, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_selftest_wait_timeout: %s", cudaGetErrorString(e));
+    return DDTREE_OK;
+}
+
 int ddtree_device_status(void) {
     uint32_t* p = device_status_word();
     if (!p) return fail(DDTREE_ERR_CUDA, "ddtree_device_status: no status word");

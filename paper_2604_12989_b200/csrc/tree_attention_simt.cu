@@ -23,6 +23,7 @@ tree_attention_f32_kernel(const float* __restrict__ q, const float* __restrict__
     constexpr int E = D / 32;  // output elements per lane
     __shared__ float s_q[kWarpsPerCta][D];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_wait();  // n_rows and the mask may come from the kernel launched just before
     const long long task = static_cast<long long>(blockIdx.x) * kWarpsPerCta + warp;
     if (task >= static_cast<long long>(R) * N * Hq) return;
     const int h = static_cast<int>(task % Hq);
@@ -109,16 +110,17 @@ cudaError_t launch_tree_attention_f32(const AttnArgs& a, cudaStream_t st) {
     const long long tasks = static_cast<long long>(a.R) * a.N * a.Hq;
     const unsigned grid = static_cast<unsigned>((tasks + kWarpsPerCta - 1) / kWarpsPerCta);
     const float scale_log2 = a.scale * kLog2e;
-#define DDTREE_LAUNCH(D)                                                                                     \
-    tree_attention_f32_kernel<D><<<grid, kWarpsPerCta * 32, 0, st>>>(                                        \
-        static_cast<const float*>(a.q), static_cast<const float*>(a.k_cache),                                \
-        static_cast<const float*>(a.v_cache), static_cast<const float*>(a.k_tree),                           \
-        static_cast<const float*>(a.v_tree), a.cu_prefix, a.anc_mask, a.n_rows, static_cast<float*>(a.out),  \
-        a.lse, a.R, a.N, a.W, a.Hq, a.Hkv, scale_log2)
-    if (a.d == 64) DDTREE_LAUNCH(64);
-    else DDTREE_LAUNCH(128);
-#undef DDTREE_LAUNCH
-    return cudaGetLastError();
+    const float* q = static_cast<const float*>(a.q);
+    const float* kc = static_cast<const float*>(a.k_cache);
+    const float* vc = static_cast<const float*>(a.v_cache);
+    const float* kt = static_cast<const float*>(a.k_tree);
+    const float* vt = static_cast<const float*>(a.v_tree);
+    float* out = static_cast<float*>(a.out);
+    if (a.d == 64)
+        return launch_pdl(tree_attention_f32_kernel<64>, dim3(grid), dim3(kWarpsPerCta * 32), 0, st, q, kc, vc, kt, vt,
+                          a.cu_prefix, a.anc_mask, a.n_rows, out, a.lse, a.R, a.N, a.W, a.Hq, a.Hkv, scale_log2);
+    return launch_pdl(tree_attention_f32_kernel<128>, dim3(grid), dim3(kWarpsPerCta * 32), 0, st, q, kc, vc, kt, vt,
+                      a.cu_prefix, a.anc_mask, a.n_rows, out, a.lse, a.R, a.N, a.W, a.Hq, a.Hkv, scale_log2);
 }
 
 }  // namespace ddtree

@@ -5,52 +5,54 @@
 // Rows of one KV head are the (node, g) pairs of its G = Hq/Hkv query heads, row = node*G + g, so
 // that budget x G rows share each K/V tile and QK^T / PV are dense 128x128x128 contractions.
 //
-// One CTA = one (request, KV head, 128-row tile, KV split).  Warp roles:
-//   warps 0-7  softmax: two threads per row (TMEM lane = row).  Thread (row, h) owns key columns
-//              [64h, 64h+64) of every KV tile with its OWN reference maximum, sum and O accumulator
-//              (O_0, O_1 in TMEM), so the halves of a row never synchronise inside the loop; at the end
-//              they are merged like two KV splits.  Exponentials (MUFU) are the co-bottleneck of this
-//              kernel, so all eight warps work on every tile
-//   warp 8     TMA producer: Q once, then separate 3-stage rings for K tiles and V tiles
-//   warp 9     MMA issuer: S = Q K^T (operands in shared memory) runs one tile ahead into two TMEM
-//              score buffers; O_h += P_h V_h (P read from TMEM, V as an MN-major shared-memory
-//              operand) as soon as half h of the tile is ready; owns the TMEM allocation
-// A last row tile of at most 16 rows (the root's G rows of a tree of 2^k nodes) takes a path of its own
-// in batches that fill the SMs several times over: see tail_tile_cta.
+// One CTA = one (request, KV head, pair of 128-row tiles A and B, KV split).  Warp roles:
+//   warps 0-3  softmax of row tile A: one thread per row (TMEM lane = row), all 128 key columns of a
+//              KV tile, read from tensor memory 64 at a time
+//   warps 4-7  softmax of row tile B, the same
+//   warp 8     TMA producer: Q_A, Q_B once, then one ring of K and V tiles (K_0, V_0, K_1, V_1, ...)
+//   warp 9     MMA issuer; owns the TMEM allocation.  Per KV tile j it issues, for A and then for B,
+//              O_X += P_X V_j followed by S_X = Q_X K_{j+1}^T: the products of one row tile run while
+//              the other row tile's threads exponentiate, so that the tensor pipe and the
+//              exponential unit, which cost the same per tile at head dim 128, overlap
+//   warp 10    clears the rows of a staged V tile that belong to no visible key (the ragged end of a
+//              prefix, tree rows past n_rows): their probabilities are zero, but 0 x NaN is not
+// Tensor memory: S_A, S_B (fp32 scores, 128 columns each; the bf16 probabilities overwrite the first
+// 64 columns of their own scores), O_A, O_B (128 columns each): all 512 columns.
+// A last row tile of at most 16 rows (the root's G rows of a tree of 2^k nodes) is a CTA of its own
+// with the roles of rows and keys swapped: see tail_tile_cta.
 // The ancestor bitmask is applied only on tree tiles; prefix tiles need at most a length test on
 // the request's last tile.  Each split writes its normalised rows (fp16) with their reference maximum
-// and sum; a combine kernel merges them by log-sum-exp.  Every wait is bounded: when one gives up, the CTA raises a flag in the
-// device status word, drains its copies and leaves without touching its outputs.
+// and sum; a combine kernel merges them by log-sum-exp.  Every wait is bounded: when one gives up, the
+// CTA raises a flag in the device status word, drains its copies and leaves without touching its outputs.
 #include "common.cuh"
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <math_constants.h>
 #include <algorithm>
 #include <mutex>
+#include <type_traits>
 #include <unordered_map>
 #include <vector>
 
 namespace ddtree {
 namespace {
 
-constexpr int kTile = 128;            // rows per CTA, keys per KV tile, head dim
-constexpr int kStages = 3;
-constexpr int kSBufs = 2;              // score buffers in TMEM: Q K^T runs one tile ahead of the softmax
-constexpr int kSoftmaxThreads = 256;   // two threads per row, 64 key columns each
-constexpr int kGroupThreads = 128;     // threads of one column half
-constexpr int kProducerWarp = 8, kMmaWarp = 9;
-constexpr int kThreads = 320;          // warps 0-7: softmax; 8: TMA producer; 9: MMA issuer
+constexpr int kTile = 128;            // rows per row tile, keys per KV tile, head dim
+constexpr int kRing = 5;              // K/V tiles in flight: K_j in slot 2j % 5, V_j in slot (2j+1) % 5
+constexpr int kProducerWarp = 8, kMmaWarp = 9, kFixWarp = 10;
+constexpr int kThreads = 384;         // warps 0-3 / 4-7: softmax A / B; 8: producer; 9: MMA; 10: V clean-up; 11: idle
 constexpr uint32_t kHalfBytes = 128 * 64 * 2;      // one 64-wide half of a 128x128 bf16 tile
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;         // S buffers at columns 0 and 128; half h's bf16 P overwrites columns [64h, 64h+32)
-constexpr uint32_t kColO = 256;       // O accumulators of the two column halves at columns 256 and 384
+constexpr uint32_t kColS = 0;         // S_X at column 128 X; P_X (bf16 pairs) in its first 64 columns
+constexpr uint32_t kColO = 256;       // O_X at column 256 + 128 X
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kMaxOrdered = 128;
 constexpr uint32_t kErrTimeout = 0x5101;
 constexpr uint32_t kErrAlign = 0x5102;
+constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // 256 x 208 + 128 x 88 = 384 x 168 registers
 
 // ---- PTX wrappers --------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -86,9 +88,9 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when it gave up (or another thread of the CTA already did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t limit) {
     if (mbar_test(bar, parity)) return true;
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 32) {
             __nanosleep(64);
@@ -97,6 +99,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     *abort_flag = 1;
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    return mbar_wait_limit(bar, parity, abort_flag, kSpinLimit);
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
@@ -115,6 +120,7 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 // One lane of a converged warp (all 32 lanes must call this together).
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
@@ -125,6 +131,10 @@ __device__ __forceinline__ bool elect_one() {
         : "=r"(pred));
     return pred != 0;
 }
+// Register budget of the calling warp group (all four warps of it execute this together).
+template <int kRegs> __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs)); }
+template <int kRegs> __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs)); }
+
 // D[tmem] (+)= A[smem desc] * B[smem desc].  The accumulate flag is a template argument and the
 // operands are "base + constant": one thread issues every MMA of the CTA, and anything beyond a
 // handful of scalar instructions per MMA makes that thread, not the tensor pipe, the bottleneck.
@@ -176,6 +186,13 @@ __device__ __forceinline__ void umma_ts(uint32_t d, uint32_t a, uint64_t b, uint
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 " DDTREE_L32 ", [%32];" : DDTREE_R32(v, o) : "r"(taddr))
 #define TMEM_ST32(taddr, v, o) \
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], " DDTREE_S32 ";" ::"r"(taddr), DDTREE_W32(v, o) : "memory")
+// 64 consecutive columns of this thread's TMEM lane -> v[0 .. 63] (one round trip: a load in flight holds the
+// warp's following instructions back, so fewer, wider loads are cheaper than several narrow ones)
+__device__ __forceinline__ void tmem_ld64(uint32_t (&v)[64], uint32_t taddr) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "=r"(v[32]), "=r"(v[33]), "=r"(v[34]), "=r"(v[35]), "=r"(v[36]), "=r"(v[37]), "=r"(v[38]), "=r"(v[39]), "=r"(v[40]), "=r"(v[41]), "=r"(v[42]), "=r"(v[43]), "=r"(v[44]), "=r"(v[45]), "=r"(v[46]), "=r"(v[47]), "=r"(v[48]), "=r"(v[49]), "=r"(v[50]), "=r"(v[51]), "=r"(v[52]), "=r"(v[53]), "=r"(v[54]), "=r"(v[55]), "=r"(v[56]), "=r"(v[57]), "=r"(v[58]), "=r"(v[59]), "=r"(v[60]), "=r"(v[61]), "=r"(v[62]), "=r"(v[63])
+                 : "r"(taddr));
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // 16 consecutive columns of this thread's TMEM lane
@@ -215,54 +232,11 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
            (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTile >> 4) << 24);
 }
 
-// Optional timeline instrumentation (compiled in only with -DDDTREE_TRACE; development aid).
-#ifdef DDTREE_TRACE
-__device__ unsigned long long* g_trace = nullptr;
-__device__ __forceinline__ void trace_mark(int idx) {
-    if (g_trace) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-        g_trace[cta * 64 + idx] = t;
-    }
-}
-#define TRACE(idx) trace_mark(idx)
-__device__ __forceinline__ void trace_clk(int idx) {
-    if (g_trace) {
-        long long t;
-        asm volatile("mov.u64 %0, %%clock64;" : "=l"(t) :: "memory");
-        const int cta = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-        g_trace[cta * 64 + idx] = static_cast<unsigned long long>(t);
-    }
-}
-#define TRACE_CLK(idx) trace_clk(idx)
-// Low-overhead time stamps: clock64 into registers for two steady-state tiles, written out once
-// after the loop (a stamp that writes to global memory costs ~300 cycles and distorts the loop).
-#ifndef DDTREE_STAMP_TILE
-#define DDTREE_STAMP_TILE 8
-#endif
-constexpr int kStampTile = DDTREE_STAMP_TILE;
-#define STAMP_DECL long long stamp_[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
-#define STAMP(cond, i) do { if (cond) { long long t_; asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_)); stamp_[i] = t_; } } while (0)
-#define STAMP_FLUSH(cond, base) do { if ((cond) && g_trace) { \
-        const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); \
-        for (int i_ = 0; i_ < 16; ++i_) if (stamp_[i_]) g_trace[cta_ * 64 + (base) + i_] = static_cast<unsigned long long>(stamp_[i_]); } } while (0)
-#else
-constexpr int kStampTile = 8;
-#define STAMP_DECL ((void)0)
-#define STAMP(cond, i) ((void)0)
-#define STAMP_FLUSH(cond, base) ((void)0)
-#define TRACE(idx) ((void)0)
-#define TRACE_CLK(idx) ((void)0)
-#endif
-
 struct Smem {
-    uint8_t q[kTileBytes];
-    uint8_t k[kStages][kTileBytes];
-    uint8_t v[kStages][kTileBytes];
-    uint64_t q_full, k_full[kStages], k_free[kStages], v_full[kStages], v_free[kStages];
-    uint64_t s_full[kSBufs], p_ready[kSBufs][2], o_done[2], fin;
-    float xm[2][kTile], xl[2][kTile]; // [column half][row]: reference maximum and sum, exchanged at the end
+    uint8_t q[2][kTileBytes];        // row tiles A and B
+    uint8_t kv[kRing][kTileBytes];
+    uint64_t q_full[2], kv_full[kRing], kv_free[kRing], v_fix[kRing];
+    uint64_t s_full[2], p_half[2], p_ready[2], o_half[2], o_final[2];
     uint32_t tmem_base;
     uint32_t abort;
 };
@@ -276,9 +250,16 @@ struct KernelParams {
     __half* part_o;  // [S, R, Hkv, rows_pad, 128]: each split's O divided by its own sum, fp16
     float2* part_ml; // [S, R, Hkv, rows_pad] (reference max in log2 units, sum)
     uint32_t* status;
-    int R, N, W, Hq, Hkv, G, splits, rows_pad;
+    int R, N, W, Hq, Hkv, G, rows_pad;
+    int full_tiles;   // 128-row tiles handled in pairs by the CTAs of the main path
+    int pairs;        // ceil(full_tiles / 2)
+    int splits;       // KV splits of a pair
+    int tail;         // 1: the last 128-row tile (index full_tiles) is a short tile with a CTA of its own
+    int tail_splits;  // KV splits of the short tile
+    int units;        // CTAs per (request, KV head) = pairs * splits + tail * tail_splits
+    int node0;        // the combine kernel covers nodes node0 .. N-1
     float scale_log2;
-    // blockIdx.z -> request, longest prefix first (CTAs are dispatched in index order: the long ones must
+    // grid index -> request, longest prefix first (CTAs are dispatched in index order: the long ones must
     // not be left for the end); identity when the batch has more than kMaxOrdered requests
     int ordered;
     uint16_t order[kMaxOrdered];
@@ -295,52 +276,80 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-// Two non-negative finite floats -> packed bf16 pair (low half = a), rounding to nearest with ties
-// away from zero: add half an ulp of bf16 to the bit pattern, keep the upper 16 bits.  Done with
-// integer adds and one byte permute so that it stays off the conversion/transcendental unit, which
-// the exponentials already saturate.
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-    return __byte_perm(__float_as_uint(a) + 0x8000u, __float_as_uint(b) + 0x8000u, 0x7632);
+// Two non-negative floats -> packed bf16 pair (low half = a), round to nearest even.
+__device__ __forceinline__ uint32_t pack_cvt(float a, float b) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
+    return r;
 }
 
-// Exponentials of score columns [kBegin, kEnd) of one thread relative to the reference m_use, packed to
-// bf16 pairs (low half = even key), and their sum added to rowsum.
-template <int kBegin, int kEnd>
-__device__ __forceinline__ void exp_block(const uint32_t (&sv)[64], uint32_t (&pk)[32], float& rowsum, float scale_log2,
-                                          float m_use) {
+// Exponentials of the 64 scores of half a tile relative to the reference m_use, packed to bf16 pairs
+// (pk[c] = keys 2c, 2c+1 of the half, c < 32); returns their sum.
+__device__ __forceinline__ float exp_pack_64(const uint32_t (&x)[64], uint32_t (&pk)[32], float scale_log2, float m_use) {
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-    for (int c = kBegin; c < kEnd; c += 2) {
-        const float e0 = ex2(fmaf(__uint_as_float(sv[c]), scale_log2, -m_use));
-        const float e1 = ex2(fmaf(__uint_as_float(sv[c + 1]), scale_log2, -m_use));
-        rowsum += e0 + e1;
-        pk[c >> 1] = pack_bf16(e0, e1);
+    for (int c = 0; c < 64; c += 4) {
+        const float e0 = ex2(fmaf(__uint_as_float(x[c]), scale_log2, -m_use));
+        const float e1 = ex2(fmaf(__uint_as_float(x[c + 1]), scale_log2, -m_use));
+        const float e2 = ex2(fmaf(__uint_as_float(x[c + 2]), scale_log2, -m_use));
+        const float e3 = ex2(fmaf(__uint_as_float(x[c + 3]), scale_log2, -m_use));
+        s0 += e0; s1 += e1; s2 += e2; s3 += e3;
+        pk[c >> 1] = pack_cvt(e0, e1);
+        pk[(c >> 1) + 1] = pack_cvt(e2, e3);
     }
+    return (s0 + s1) + (s2 + s3);
 }
 
-// Replace the scores of invisible keys by -inf: bit c of `word` tells whether key c of this
-// 32-key group is visible to this row.
-__device__ __forceinline__ void mask32(uint32_t (&sv)[64], int o, uint32_t word) {
+__device__ __forceinline__ float max_64(const uint32_t (&x)[64]) {
+    float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+    for (int c = 0; c < 64; c += 8)
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            mx4[k] = max3(mx4[k], __uint_as_float(x[c + 2 * k]), __uint_as_float(x[c + 2 * k + 1]));
+    return fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]);
+}
+
+// Replace the scores of invisible keys by -inf: bit c of `word` tells whether key o + c is visible to this row.
+template <int kN>
+__device__ __forceinline__ void mask32(uint32_t (&sv)[kN], int o, uint32_t word) {
 #pragma unroll
     for (int c = 0; c < 32; ++c)
         if (!((word >> c) & 1u)) sv[o + c] = 0xff800000u;
 }
 
+// Number of keys of KV tile t (absolute index within the request) that any row may see: the rows of a
+// staged V tile from there on belong to another request, to padding or to nobody.
+__device__ __forceinline__ int keys_in_tile(int t, int prefix_tiles, int P, int n) {
+    return t < prefix_tiles ? min(kTile, P - t * kTile) : min(kTile, n - (t - prefix_tiles) * kTile);
+}
+// Zero rows [first, 128) of a staged V tile (both 64-wide halves; the 128-byte swizzle permutes 16-byte
+// chunks inside a row only).  Whole warp; the writes are made visible to the tensor pipe.
+__device__ __forceinline__ void clear_v_rows(uint8_t* tile, int first, int lane) {
+    const int chunks = (kTile - first) * 16;
+    for (int i = lane; i < chunks; i += 32) {
+        const int row = first + (i >> 4), c = i & 15;
+        *reinterpret_cast<uint4*>(tile + (c >> 3) * kHalfBytes + row * 128 + (c & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    fence_async_smem();
+    __syncwarp();
+}
+
 // ---- short last row tile ----------------------------------------------------------------------
 // A tree of B = 2^k nodes plus the root leaves G rows over for a last row tile of their own; run
-// through the path below, that tile would cost as much as a full one (a fifth of all CTAs for B = 128,
-// G = 4).  With so few rows the roles of
+// through the main path, that tile would cost as much as a full one.  With so few rows the roles of
 // rows and keys are swapped for the scores: S^T = K Q^T puts the 128 keys of a tile on the TMEM lanes
 // and the (at most 16) rows on the columns, so a thread exponentiates 16 values per tile instead of
-// 64, keeps its own partial row sums, and the tile costs little more than the copy of its K/V.  The
+// 128, keeps its own partial row sums, and the tile costs little more than the copy of its K/V.  The
 // second product is swapped as well: O^T += V^T P^T with the V tile as the 128-row (MN-major) operand
 // and P^T, 16 rows x 128 keys written to shared memory by the key threads, as the narrow one; O^T
 // has the head dimension on the lanes and one column per row.  A row's reference maximum is set by
 // an exact reduction over the key threads on the first tile and whenever an exponential exceeds
 // 2^24; otherwise the threads only meet at one barrier per tile.  Two groups of 128 key threads take
-// alternate tiles, each with its own reference maxima, sums and O^T, merged at the end.  The CTA sees
-// the whole KV range of its rows (the path is used only where there are no KV splits) and writes the
-// output itself.  Measured: ~1200 cycles per KV tile against ~2200 on the full-tile path; the tensor
-// pipe is the limit (16 instructions per tile that each stream a 4 KB operand from shared memory).
+// alternate tiles, each with its own reference maxima, sums and O^T, merged at the end.  The CTA walks
+// its KV split of the request and writes the output itself, or its normalised partial rows when the
+// short tile's KV range is split.  Measured: ~1200 cycles per KV tile; the tensor pipe is the limit
+// (16 instructions per tile that each stream a 4 KB operand from shared memory).
 constexpr int kTailRows = 16;
 constexpr int kTailKStages = 3, kTailVStages = 3;
 constexpr uint32_t kTailQHalf = kTailRows * 128;  // one 64-wide half of the 16-row Q or P^T tile
@@ -354,6 +363,7 @@ struct TailSmem {
     uint8_t q[2 * kTailQHalf];      // the tile's 16 query rows
     uint8_t pt[2][2][2 * kTailQHalf];  // [group][buffer] P^T: [row][key], two 64-key halves, 128-byte swizzle (K-major operand)
     uint64_t q_full, k_full[kTailKStages], k_free[kTailKStages], v_full[kTailVStages], v_free[kTailVStages];
+    uint64_t v_fix[kTailVStages];
     // One barrier per buffer, each watched by one key group only: a parity wait must see every phase in turn.
     uint64_t s_full[kTailSBufs], p_ready[2][2], o_done[2][2];
     float red[2][4][kTailRows];  // [group][warp]: row maxima inside the loop, row sums at the end
@@ -363,19 +373,27 @@ struct TailSmem {
     uint32_t key_fail[2];  // per group: a key thread's wait gave up (written before, read after a barrier of the group)
 };
 
-__device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const CUtensorMap* map_kc, const CUtensorMap* map_vc,
+__device__ __noinline__ void tail_tile_cta(const CUtensorMap* map_qt, const CUtensorMap* map_kc, const CUtensorMap* map_vc,
                                               const CUtensorMap* map_kt, const CUtensorMap* map_vt, const KernelParams& p,
-                                              uint8_t* smem_raw, int kvh, int rt, int r, int n) {
+                                              uint8_t* smem_raw, int kvh, int r, int n, int split) {
     TailSmem& sm = *reinterpret_cast<TailSmem*>(smem_raw);
+    const int rt = p.full_tiles;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rows = min(n * p.G - rt * kTile, kTailRows);  // valid rows of this tile (> 0: checked by the caller)
     const int p0 = p.cu_prefix[r], P = p.cu_prefix[r + 1] - p0;
     const int prefix_tiles = (P + kTile - 1) / kTile, tree_tiles = (n + kTile - 1) / kTile;
-    const int my_tiles = prefix_tiles + tree_tiles;  // the whole KV range (this path runs without KV splits), >= 1
-    constexpr int t_begin = 0;
+    const int tiles = prefix_tiles + tree_tiles;
+    const int per = (tiles + p.tail_splits - 1) / p.tail_splits;
+    const int t_begin = split * per;
+    const int my_tiles = max(0, min(tiles, t_begin + per) - t_begin);
+    const bool direct = p.tail_splits == 1;
+    const size_t part_row0 = ((static_cast<size_t>(split) * p.R + r) * p.Hkv + kvh) * p.rows_pad + rt * kTile;
+    if (my_tiles == 0) {  // this split has nothing to do for this request: publish empty partials
+        if (tid < rows) p.part_ml[part_row0 + tid] = make_float2(-CUDART_INF_F, 0.f);
+        return;
+    }
 
     volatile uint32_t* abort_flag = &sm.abort;
-    if (tid == 0) TRACE(60);
     int k_issued = 0, v_issued = 0;
     auto tile_row = [&](int j, bool& in_prefix) {
         const int t = t_begin + j;
@@ -399,14 +417,18 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
     if (warp == kProducerWarp && lane == 0) {
         mbar_init(smem_u32(&sm.q_full), 1);
         for (int s = 0; s < kTailKStages; ++s) { mbar_init(smem_u32(&sm.k_full[s]), 1); mbar_init(smem_u32(&sm.k_free[s]), 1); }
-        for (int s = 0; s < kTailVStages; ++s) { mbar_init(smem_u32(&sm.v_full[s]), 1); mbar_init(smem_u32(&sm.v_free[s]), 1); }
+        for (int s = 0; s < kTailVStages; ++s) {
+            mbar_init(smem_u32(&sm.v_full[s]), 1);
+            mbar_init(smem_u32(&sm.v_free[s]), 1);
+            mbar_init(smem_u32(&sm.v_fix[s]), 1);
+        }
         for (int b = 0; b < kTailSBufs; ++b) mbar_init(smem_u32(&sm.s_full[b]), 1);
         for (int b = 0; b < 4; ++b) { mbar_init(smem_u32(&sm.p_ready[0][0]) + 8 * b, 1); mbar_init(smem_u32(&sm.o_done[0][0]) + 8 * b, 1); }
         sm.abort = 0;
         sm.key_fail[0] = 0;
         sm.key_fail[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fence_async_smem();
         const int nodes_per_tile = kTile / p.G;
         mbar_expect_tx(smem_u32(&sm.q_full), 2 * kTailQHalf);
         for (int h = 0; h < 2; ++h)
@@ -423,7 +445,7 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
         uint4* z = reinterpret_cast<uint4*>(sm.pt);
 #pragma unroll
         for (int u = 0; u < 4; ++u) z[tid + 256 * u] = make_uint4(0u, 0u, 0u, 0u);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fence_async_smem();
     }
     tc_fence_before();
     __syncthreads();
@@ -451,6 +473,17 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
                 if (++idle > kSpinLimit) { *abort_flag = 1; break; }
                 if ((idle & 255u) == 0 && *abort_flag) break;
             }
+        }
+    } else if (warp == kFixWarp) {
+        // Every staged V tile passes through this warp on its way to the MMA warp: rows that no row may see
+        // (ragged end of the prefix, tree rows past n_rows) are cleared before the product reads them; their
+        // probabilities are zero, but 0 x NaN is not.  The copies run tiles ahead, so the relay costs nothing.
+        for (int j = 0; j < my_tiles; ++j) {
+            const int s = j % kTailVStages;
+            if (!__all_sync(kFull, mbar_wait(smem_u32(&sm.v_full[s]), (j / kTailVStages) & 1, abort_flag))) break;
+            const int first = keys_in_tile(t_begin + j, prefix_tiles, P, n);
+            if (first < kTile) clear_v_rows(sm.v[s], first, lane);
+            if (lane == 0) mbar_arrive(smem_u32(&sm.v_fix[s]));
         }
     } else if (warp == kMmaWarp) {
         constexpr uint32_t idesc_st = instr_desc(kTailRows, false);          // 128 keys x 16 rows, both operands K-major
@@ -487,7 +520,6 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
             if (elect_one()) issue_st(j);
             __syncwarp();
         }
-        STAMP_DECL;
         for (int j = 0; j < my_tiles && ok; ++j) {
             // One burst per tile: O_g^T += V_j^T P_j^T, then the scores of tile j+4 into the S^T buffer the key
             // threads have just read.  Every instruction streams a 128-row operand (4 KB) from shared
@@ -495,18 +527,15 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
             // ~850 cycles; the barriers are tested together beforehand to keep it from draining.
             const int s = j % kTailVStages, g = j & 1, b = (j >> 1) & 1;  // key group and its P^T buffer
             const bool more = j + kTailSBufs < my_tiles;
-            [[maybe_unused]] const bool st8 = j == kStampTile;
-            STAMP(st8, 0);
             const bool k_ok = !more || mbar_test(smem_u32(&sm.k_full[(j + kTailSBufs) % kTailKStages]), ((j + kTailSBufs) / kTailKStages) & 1);
-            const bool ready = mbar_test(smem_u32(&sm.v_full[s]), (j / kTailVStages) & 1) & k_ok &
+            const bool ready = mbar_test(smem_u32(&sm.v_fix[s]), (j / kTailVStages) & 1) & k_ok &
                                mbar_test(smem_u32(&sm.p_ready[g][b]), (j >> 2) & 1);
             if (!__all_sync(kFull, ready)) {
-                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.v_full[s]), (j / kTailVStages) & 1, abort_flag)) &&
+                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.v_fix[s]), (j / kTailVStages) & 1, abort_flag)) &&
                      (!more || wait_k(j + kTailSBufs)) &&
                      __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[g][b]), (j >> 2) & 1, abort_flag));
                 if (!ok) break;
             }
-            STAMP(st8, 1);
             tc_fence_after();
             const uint64_t vd = v_desc0 + static_cast<uint64_t>(s) * (kTileBytes >> 4);
             const uint64_t pd = p_desc0 + static_cast<uint64_t>(g * 2 + b) * ((2 * kTailQHalf) >> 4);
@@ -527,14 +556,12 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
                 if (more) issue_st(j + kTailSBufs);
             }
             __syncwarp();
-            STAMP(st8, 2);
         }
-        STAMP_FLUSH(lane == 0, 0);
-    } else {
+    } else if (warp < 8) {
         // ---- key threads: two groups of 128 (warps 0-3: even tiles, warps 4-7: odd tiles).  Thread c of a
         //      group owns key c of its tiles and head-dim element c of the group's O^T.  A group has its own
-        //      reference maxima, sums and O^T, like the column halves of the full tiles: the groups never
-        //      talk inside the loop and are merged at the end like two KV splits. ----------------------
+        //      reference maxima, sums and O^T: the groups never talk inside the loop and are merged at the
+        //      end like two KV splits. ------------------------------------------------------------------
         const int g = warp >> 2, c = tid & (kTile - 1);
         const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         const uint32_t o_addr = lane_addr + kColOT + g * 32;
@@ -550,24 +577,16 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
             for (int i = 0; i < kTailRows; ++i)
                 if (i < rows)
                     *reinterpret_cast<__nv_bfloat16*>(base + i * 128 + ((chunk ^ (i & 7)) << 4)) = __float2bfloat16_rn(pv[i]);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            fence_async_smem();
         };
         // completion of the product of this group's q-th tile (it read P^T[q % 2] and added to the group's O^T)
         auto wait_pv = [&](int q) {
             return __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[g][q & 1]), (q >> 1) & 1, abort_flag));
         };
         bool failed = false;
-        STAMP_DECL;
         for (int q = 0; q < my_count; ++q) {
             const int j = 2 * q + g, t = t_begin + j, b = q & 1, sb = j % kTailSBufs;
-            [[maybe_unused]] const bool st8 = j == kStampTile;
-            STAMP(st8, 0);
-            STAMP(j == kStampTile + 2, 8);
-            STAMP(j == kStampTile + 8, 9);
-            STAMP(q == 0, 10);
-            STAMP(q == 4, 12);
             bool ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.s_full[sb]), (j / kTailSBufs) & 1, abort_flag));
-            STAMP(st8, 1);
             uint32_t sv[kTailRows];
 #pragma unroll
             for (int i = 0; i < kTailRows; ++i) sv[i] = 0u;
@@ -594,7 +613,6 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
             }
             tmem_wait_ld();
             tc_fence_before();
-            STAMP(st8, 2);
             float x[kTailRows], pv[kTailRows];
             bool need = false;
 #pragma unroll
@@ -603,17 +621,13 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
                 pv[i] = ex2(x[i] - (mref[i] == -CUDART_INF_F ? 0.f : mref[i]));
                 if (i < rows) need |= mref[i] == -CUDART_INF_F || !(pv[i] < 16777216.f);
             }
-            STAMP(st8, 3);
             // P^T[b] was read by the product of this group's tile q-2
             if (ok && q > 1) ok = wait_pv(q - 2);
-            STAMP(st8, 4);
             store_p(b, pv);
-            STAMP(st8, 5);
             // A wait that gave up joins the vote, and the flag it left is read only after the barrier: every
             // thread of the group takes the same way out (a thread missing at a later barrier would hang the others).
             if (!ok) sm.key_fail[g] = 1;
             const bool slow = bar_keys_or(g, need || !ok);
-            STAMP(st8, 6);
             if (slow) {
                 if (*reinterpret_cast<volatile uint32_t*>(&sm.key_fail[g])) { failed = true; break; }
 #pragma unroll
@@ -657,10 +671,7 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
 #pragma unroll
             for (int i = 0; i < kTailRows; ++i) l_part[i] += pv[i];
             if (c == 0) mbar_arrive(smem_u32(&sm.p_ready[g][b]));
-            STAMP(st8, 7);
         }
-        STAMP(true, 11);
-        STAMP_FLUSH(c == 0, g ? 32 : 16);
 
         // ---- epilogue: row sums over each group's threads, then group 0 merges the two groups and thread c
         //      writes head-dim element c of every row ----------------------------------------------------
@@ -700,10 +711,15 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
                         const float f = l_row > 0.f ? 1.f / l_row : 0.f;
                         float o = __uint_as_float(oa[i]) * (w_a * f);
                         if (w_b > 0.f) o = fmaf(__uint_as_float(ob[i]), w_b * f, o);
-                        const int grow = rt * kTile + i, node = grow / p.G;
-                        const size_t head_row = (static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + grow % p.G;
-                        p.out[head_row * kTile + c] = __float2bfloat16_rn(o);
-                        if (c == 0 && p.lse) p.lse[head_row] = (m_row + log2f(l_row)) / kLog2e;
+                        if (direct) {
+                            const int grow = rt * kTile + i, node = grow / p.G;
+                            const size_t head_row = (static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + grow % p.G;
+                            p.out[head_row * kTile + c] = __float2bfloat16_rn(o);
+                            if (c == 0 && p.lse) p.lse[head_row] = (m_row + log2f(l_row)) / kLog2e;
+                        } else {
+                            p.part_o[(part_row0 + i) * kTile + c] = __float2half_rn(o);
+                            if (c == 0) p.part_ml[part_row0 + i] = make_float2(m_row, l_row);
+                        }
                     }
                 }
             }
@@ -713,7 +729,6 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
     // ---- teardown -------------------------------------------------------------------------------
     tc_fence_before();
     __syncthreads();
-    if (tid == 0) TRACE(61);
     if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -732,15 +747,37 @@ __device__ __forceinline__ void tail_tile_cta(const CUtensorMap* map_qt, const C
     }
 }
 
-// kShortTile: the grid's last row tile takes the short-tile path.  A kernel of its own rather than a run-time
-// flag: with that path compiled in, a layer of a one-request batch (CTAs that live ~10 us) was measured
-// ~2 us slower although none of its CTAs takes the path, and such batches never use it.
-template <bool kShortTile>
+// ---- main path: softmax of one KV tile by one thread (row) ----------------------------------------
+// Visibility of the 128 keys of tile t to a row: vis[w] has bit c set iff key 32 w + c is visible.
+// Returns true when all 128 are (no masking needed).
+__device__ __forceinline__ bool tile_visibility(uint32_t (&vis)[4], int t, int prefix_tiles, int P, int W, bool valid,
+                                                const uint32_t* mrow) {
+    bool all_visible = false;
+    if (!valid) {
+#pragma unroll
+        for (int w = 0; w < 4; ++w) vis[w] = 0u;
+    } else if (t < prefix_tiles) {
+        const int left = P - t * kTile;  // keys of this request in the tile
+        all_visible = left >= kTile;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const int lw = left - 32 * w;
+            vis[w] = lw >= 32 ? kFull : (lw <= 0 ? 0u : ((1u << lw) - 1u));
+        }
+    } else {
+        const int w0 = (t - prefix_tiles) * 4;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) vis[w] = w0 + w < W ? mrow[w0 + w] : 0u;
+    }
+    return all_visible;
+}
+
+template <bool kTail>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kc,
                            const __grid_constant__ CUtensorMap map_vc, const __grid_constant__ CUtensorMap map_kt,
                            const __grid_constant__ CUtensorMap map_vt, const __grid_constant__ CUtensorMap map_qt,
-                           const KernelParams p) {
+                           const __grid_constant__ KernelParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
     if (smem_u32(smem_raw) & 1023u) {  // the 128-byte swizzle needs 1024-byte aligned tiles
@@ -749,17 +786,23 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     }
 
     pdl_wait();               // everything read below may come from the previous kernel of the stream
-    const int split = blockIdx.x;
-    const int kvh = blockIdx.y % p.Hkv, rt = blockIdx.y / p.Hkv;
-    const int r = p.ordered ? p.order[blockIdx.z] : blockIdx.z;
+    const int unit = blockIdx.x % p.units;
+    const int kvh = (blockIdx.x / p.units) % p.Hkv;
+    const int zr = blockIdx.x / (p.units * p.Hkv);
+    const int r = p.ordered ? p.order[zr] : zr;
     const int n = min(p.n_rows[r], p.N);
-    if (rt * kTile >= n * p.G) return;  // whole row tile is padding
-    if constexpr (kShortTile) {
-        if (rt == p.rows_pad / kTile - 1) {
-            tail_tile_cta(&map_qt, &map_kc, &map_vc, &map_kt, &map_vt, p, smem_raw, kvh, rt, r, n);
+    const int rows_total = n * p.G;
+    if constexpr (kTail) {
+        if (unit >= p.pairs * p.splits) {
+            if (p.full_tiles * kTile < rows_total)
+                tail_tile_cta(&map_qt, &map_kc, &map_vc, &map_kt, &map_vt, p, smem_raw, kvh, r, n, unit - p.pairs * p.splits);
             return;
         }
     }
+    const int pair = unit / p.splits, split = unit % p.splits;
+    const int rt0 = 2 * pair;
+    if (rt0 * kTile >= rows_total) return;  // the whole pair is padding
+    const bool has_b = rt0 + 1 < p.full_tiles && (rt0 + 1) * kTile < rows_total;
     const int p0 = p.cu_prefix[r], P = p.cu_prefix[r + 1] - p0;
     const int prefix_tiles = (P + kTile - 1) / kTile, tree_tiles = (n + kTile - 1) / kTile;
     const int tiles = prefix_tiles + tree_tiles;
@@ -768,64 +811,57 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     const int my_tiles = max(0, t_end - t_begin);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) TRACE(0);
-    const size_t part_row0 = ((static_cast<size_t>(split) * p.R + r) * p.Hkv + kvh) * p.rows_pad + rt * kTile;
+    const size_t part_row0 = ((static_cast<size_t>(split) * p.R + r) * p.Hkv + kvh) * p.rows_pad + rt0 * kTile;
 
     if (my_tiles == 0) {  // this split has nothing to do for this request: publish empty partials
-        if (tid < kTile) p.part_ml[part_row0 + tid] = make_float2(-CUDART_INF_F, 0.f);
+        if (tid < (has_b ? 2 : 1) * kTile) p.part_ml[part_row0 + tid] = make_float2(-CUDART_INF_F, 0.f);
         return;
     }
 
     // ---- set-up: the producer initialises the barriers and starts the first copies at once ----
     volatile uint32_t* abort_flag = &sm.abort;
-    int k_issued = 0, v_issued = 0;  // tiles whose K / V copies were started (producer lane only)
-    auto tile_row = [&](int j, bool& in_prefix) {
-        const int t = t_begin + j;
-        in_prefix = t < prefix_tiles;
-        return in_prefix ? p0 + t * kTile : r * p.N + (t - prefix_tiles) * kTile;
-    };
-    auto load_k = [&](int j) {
-        bool in_prefix;
-        const int row = tile_row(j, in_prefix), s = j % kStages;
-        mbar_expect_tx(smem_u32(&sm.k_full[s]), kTileBytes);
+    int issued = 0;  // ring units whose copy was started (producer lane only): unit u = K (u even) or V (u odd) of tile u/2
+    const int units_total = 2 * my_tiles;
+    auto load_unit = [&](int u) {
+        const int t = t_begin + (u >> 1), s = u % kRing;
+        const bool in_prefix = t < prefix_tiles;
+        const int row = in_prefix ? p0 + t * kTile : r * p.N + (t - prefix_tiles) * kTile;
+        const CUtensorMap* map = (u & 1) ? (in_prefix ? &map_vc : &map_vt) : (in_prefix ? &map_kc : &map_kt);
+        mbar_expect_tx(smem_u32(&sm.kv_full[s]), kTileBytes);
         for (int h = 0; h < 2; ++h)
-            tma_load_3d(smem_u32(sm.k[s]) + h * kHalfBytes, in_prefix ? &map_kc : &map_kt, smem_u32(&sm.k_full[s]),
-                        h * 64, kvh, row);
-    };
-    auto load_v = [&](int j) {
-        bool in_prefix;
-        const int row = tile_row(j, in_prefix), s = j % kStages;
-        mbar_expect_tx(smem_u32(&sm.v_full[s]), kTileBytes);
-        for (int h = 0; h < 2; ++h)
-            tma_load_3d(smem_u32(sm.v[s]) + h * kHalfBytes, in_prefix ? &map_vc : &map_vt, smem_u32(&sm.v_full[s]),
-                        h * 64, kvh, row);
+            tma_load_3d(smem_u32(sm.kv[s]) + h * kHalfBytes, map, smem_u32(&sm.kv_full[s]), h * 64, kvh, row);
     };
     if (warp == kProducerWarp && lane == 0) {
-        mbar_init(smem_u32(&sm.q_full), 1);
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&sm.k_full[s]), 1);
-            mbar_init(smem_u32(&sm.k_free[s]), 1);
-            mbar_init(smem_u32(&sm.v_full[s]), 1);
-            mbar_init(smem_u32(&sm.v_free[s]), 1);
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(smem_u32(&sm.q_full[x]), 1);
+            mbar_init(smem_u32(&sm.s_full[x]), 1);
+            mbar_init(smem_u32(&sm.p_half[x]), kTile);
+            mbar_init(smem_u32(&sm.p_ready[x]), kTile);
+            mbar_init(smem_u32(&sm.o_half[x]), 1);
+            mbar_init(smem_u32(&sm.o_final[x]), 1);
         }
-        for (int b = 0; b < kSBufs; ++b) {
-            mbar_init(smem_u32(&sm.s_full[b]), 1);
-            mbar_init(smem_u32(&sm.p_ready[b][0]), kGroupThreads);
-            mbar_init(smem_u32(&sm.p_ready[b][1]), kGroupThreads);
+        for (int s = 0; s < kRing; ++s) {
+            mbar_init(smem_u32(&sm.kv_full[s]), 1);
+            mbar_init(smem_u32(&sm.kv_free[s]), 1);
+            mbar_init(smem_u32(&sm.v_fix[s]), 1);
         }
-        for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&sm.o_done[b]), 1);
-        mbar_init(smem_u32(&sm.fin), kSoftmaxThreads);
         sm.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fence_async_smem();
         const int nodes_per_tile = kTile / p.G;
-        mbar_expect_tx(smem_u32(&sm.q_full), kTileBytes);
+        // Q_A, then the first K tile (the first product needs both), then Q_B and the rest of the ring
+        mbar_expect_tx(smem_u32(&sm.q_full[0]), kTileBytes);
         for (int h = 0; h < 2; ++h)
-            tma_load_4d(smem_u32(sm.q) + h * kHalfBytes, &map_q, smem_u32(&sm.q_full), h * 64, 0, kvh,
-                        r * p.N + rt * nodes_per_tile);
-        // K tiles first (the first MMAs need them), then the V tiles
-        for (; k_issued < my_tiles && k_issued < kStages; ++k_issued) load_k(k_issued);
-        for (; v_issued < my_tiles && v_issued < kStages; ++v_issued) load_v(v_issued);
+            tma_load_4d(smem_u32(sm.q[0]) + h * kHalfBytes, &map_q, smem_u32(&sm.q_full[0]), h * 64, 0, kvh,
+                        r * p.N + rt0 * nodes_per_tile);
+        load_unit(issued++);
+        if (has_b) {
+            mbar_expect_tx(smem_u32(&sm.q_full[1]), kTileBytes);
+            for (int h = 0; h < 2; ++h)
+                tma_load_4d(smem_u32(sm.q[1]) + h * kHalfBytes, &map_q, smem_u32(&sm.q_full[1]), h * 64, 0, kvh,
+                            r * p.N + (rt0 + 1) * nodes_per_tile);
+        }
+        for (; issued < units_total && issued < kRing; ++issued) load_unit(issued);
     }
     if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
@@ -836,383 +872,248 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
-    if (tid == 0) TRACE(1);
 
-    if (warp == kProducerWarp) {
-        // ---- TMA producer: K ring (freed when Q K^T has read it) and V ring (freed after P V) ---
-        if (lane == 0) {
-            while (k_issued < my_tiles || v_issued < my_tiles) {
-                if (k_issued < my_tiles) {
-                    if (!mbar_wait(smem_u32(&sm.k_free[k_issued % kStages]), ((k_issued / kStages) - 1) & 1, abort_flag)) break;
-                    load_k(k_issued++);
-                }
-                if (v_issued < my_tiles && v_issued < k_issued) {
-                    if (!mbar_wait(smem_u32(&sm.v_free[v_issued % kStages]), ((v_issued / kStages) - 1) & 1, abort_flag)) break;
-                    load_v(v_issued++);
+    if (warp >= 8) {
+        regs_dec<kRegsOther>();
+        if (warp == kProducerWarp) {
+            // ---- TMA producer: a slot is free again when the product that read it last has completed ----
+            if (lane == 0) {
+                while (issued < units_total) {
+                    if (!mbar_wait(smem_u32(&sm.kv_free[issued % kRing]), ((issued / kRing) - 1) & 1, abort_flag)) break;
+                    load_unit(issued++);
                 }
             }
-        }
-    } else if (warp == kMmaWarp) {
-        // ---- MMA issuer: the whole warp walks the loop (so that addresses live in uniform
-        //      registers) and one elected lane issues; Q K^T runs kSBufs tiles ahead of the softmax ----
-        constexpr uint32_t idesc_qk = instr_desc(kTile, false);
-        constexpr uint32_t idesc_pv = instr_desc(kTile, true);
-        const uint64_t q_desc = smem_desc(smem_u32(sm.q), 16);
-        const uint64_t k_desc0 = smem_desc(smem_u32(sm.k[0]), 16);
-        const uint64_t v_desc0 = smem_desc(smem_u32(sm.v[0]), kHalfBytes);
-        // S[j % kSBufs] = Q K_j^T: 16 head-dim elements (32 bytes) per instruction; the second 64-wide
-        // half of the tiles sits 16 KB further.  Called by the elected lane only.
-        auto issue_qk = [&](int j) {
-            const int s = j % kStages, b = j % kSBufs;
-            const uint64_t kd = k_desc0 + static_cast<uint64_t>(s) * (kTileBytes >> 4);
-            const uint32_t d_s = tmem + kColS + b * kTile;
-            if (j < 6) TRACE(30 + j);
-            umma_ss<false>(d_s, q_desc, kd, idesc_qk);
-            umma_ss<true>(d_s, q_desc + 2, kd + 2, idesc_qk);
-            umma_ss<true>(d_s, q_desc + 4, kd + 4, idesc_qk);
-            umma_ss<true>(d_s, q_desc + 6, kd + 6, idesc_qk);
-            umma_ss<true>(d_s, q_desc + 1024, kd + 1024, idesc_qk);
-            umma_ss<true>(d_s, q_desc + 1026, kd + 1026, idesc_qk);
-            umma_ss<true>(d_s, q_desc + 1028, kd + 1028, idesc_qk);
-            umma_ss<true>(d_s, q_desc + 1030, kd + 1030, idesc_qk);
-            tc_commit(smem_u32(&sm.k_free[s]));
-            tc_commit(smem_u32(&sm.s_full[b]));
-        };
-        auto wait_k = [&](int j) {
-            return __all_sync(kFull, mbar_wait(smem_u32(&sm.k_full[j % kStages]), (j / kStages) & 1, abort_flag));
-        };
-        bool ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.q_full), 0, abort_flag));
-        if (lane == 0) TRACE(2);
-        for (int j = 0; j < my_tiles && j < kSBufs && ok; ++j) {
-            ok = wait_k(j);
-            if (!ok) break;
-            tc_fence_after();
-            if (elect_one()) issue_qk(j);
-            __syncwarp();
-        }
-        STAMP_DECL;
-        for (int j = 0; j < my_tiles && ok; ++j) {
-            [[maybe_unused]] const bool st8 = j == kStampTile, st9 = j == kStampTile + 1;
-            STAMP(st8 || st9, st8 ? 0 : 3);
-            // One burst per tile: O_h += P_h V_h for both column halves of tile j, then the scores of
-            // tile j+2 into the S buffer those P halves sat in.  The tensor pipe pays a start-up
-            // latency of a few hundred cycles whenever it has drained, so bursts are kept long.
-            const int s = j % kStages, b = j % kSBufs;
-            const bool more = j + kSBufs < my_tiles;
-            // the four tests are independent instructions: their latencies overlap, and the tensor pipe
-            // drains within ~150 cycles of the last issue, so this check must be short
-            const bool k_ok = !more || mbar_test(smem_u32(&sm.k_full[(j + kSBufs) % kStages]), ((j + kSBufs) / kStages) & 1);
-            const bool ready = mbar_test(smem_u32(&sm.v_full[s]), (j / kStages) & 1) & k_ok &
-                               mbar_test(smem_u32(&sm.p_ready[b][0]), (j / kSBufs) & 1) &
-                               mbar_test(smem_u32(&sm.p_ready[b][1]), (j / kSBufs) & 1);
-            if (!__all_sync(kFull, ready)) {
-                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.v_full[s]), (j / kStages) & 1, abort_flag)) &&
-                     (!more || wait_k(j + kSBufs)) &&
-                     __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[b][0]), (j / kSBufs) & 1, abort_flag)) &&
-                     __all_sync(kFull, mbar_wait(smem_u32(&sm.p_ready[b][1]), (j / kSBufs) & 1, abort_flag));
-                if (!ok) break;
+        } else if (warp == kFixWarp) {
+            // ---- V clean-up: every staged V tile passes through this warp on its way to the MMA warp; rows
+            //      that no row may see are cleared (see clear_v_rows).  The copies run tiles ahead of the
+            //      products, so the relay is off the critical path. ----
+            for (int j = 0; j < my_tiles; ++j) {
+                const int u = 2 * j + 1, s = u % kRing;
+                if (!__all_sync(kFull, mbar_wait(smem_u32(&sm.kv_full[s]), (u / kRing) & 1, abort_flag))) break;
+                const int first = keys_in_tile(t_begin + j, prefix_tiles, P, n);
+                if (first < kTile) clear_v_rows(sm.kv[s], first, lane);
+                if (lane == 0) mbar_arrive(smem_u32(&sm.v_fix[s]));
             }
-            STAMP(st8 || st9, st8 ? 1 : 4);
-            tc_fence_after();
-            const uint64_t vd = v_desc0 + static_cast<uint64_t>(s) * (kTileBytes >> 4);
-            const uint32_t a_p = tmem + kColS + b * kTile;  // bf16 P: half h in columns [64h, 64h+32)
-            if (elect_one()) {
-                if (j < 5) TRACE(36 + 2 * j);
-                // 16 keys (16 rows of 128 bytes) per instruction; half h covers keys [64h, 64h+64) of the tile
-                if (j > 0) umma_ts<true>(tmem + kColO, a_p, vd, idesc_pv);
-                else umma_ts<false>(tmem + kColO, a_p, vd, idesc_pv);
-                umma_ts<true>(tmem + kColO, a_p + 8, vd + 128, idesc_pv);
-                umma_ts<true>(tmem + kColO, a_p + 16, vd + 256, idesc_pv);
-                umma_ts<true>(tmem + kColO, a_p + 24, vd + 384, idesc_pv);
-                tc_commit(smem_u32(&sm.o_done[0]));
-                if (j > 0) umma_ts<true>(tmem + kColO + kTile, a_p + 64, vd + 512, idesc_pv);
-                else umma_ts<false>(tmem + kColO + kTile, a_p + 64, vd + 512, idesc_pv);
-                umma_ts<true>(tmem + kColO + kTile, a_p + 72, vd + 640, idesc_pv);
-                umma_ts<true>(tmem + kColO + kTile, a_p + 80, vd + 768, idesc_pv);
-                umma_ts<true>(tmem + kColO + kTile, a_p + 88, vd + 896, idesc_pv);
-                tc_commit(smem_u32(&sm.o_done[1]));
-                tc_commit(smem_u32(&sm.v_free[s]));
-                if (more) issue_qk(j + kSBufs);
-            }
-            __syncwarp();
-            STAMP(st8 || st9, st8 ? 2 : 5);
-        }
-        STAMP_FLUSH(lane == 0, 0);
-    } else {
-        // ---- softmax: 256 threads; thread (wt, half) owns key columns [64*half, 64*half+64) of row wt in
-        //      every tile, with its own reference maximum, sum and O accumulator: the two halves of a
-        //      row never talk until the end, where they are merged like two KV splits -----------------
-        const int half = tid >> 7, wt = tid & (kTile - 1);
-        const int grow = rt * kTile + wt;           // row among this KV head's rows
-        const int node = grow / p.G;
-        const bool valid = node < n;
-        const uint32_t* mrow = p.anc_mask + (static_cast<size_t>(r) * p.N + (valid ? node : 0)) * p.W;
-        const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        const uint32_t o_addr = lane_addr + kColO + half * kTile;
-        float m_run = -CUDART_INF_F;   // reference maximum of the exponentials, scaled log2 units
-        float l_run = 0.f;
-        bool ok = true;
-        bool s_ready = false;    // result of the early test of s_full for the coming tile
-        bool preloaded = false;  // the TMEM load of the coming tile's scores is already in flight
-        uint32_t sv[64];
-        STAMP_DECL;
-        // ---- first tile, outside the loop: there is no reference maximum yet, so the exact maximum comes
-        //      first and the exponentials are taken once (inside the loop the first tile would take the
-        //      optimistic pass and then the revisit: twice the exponentials, ~0.6 us per CTA) ----------------
-        {
-            const uint32_t s_addr = lane_addr + kColS + half * 64;
-            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.s_full[0]), 0, abort_flag));
+        } else if (warp == kMmaWarp) {
+            // ---- MMA issuer: the whole warp walks the loop (so that addresses live in uniform registers)
+            //      and one elected lane issues ----
+            constexpr uint32_t idesc_qk = instr_desc(kTile, false);
+            constexpr uint32_t idesc_pv = instr_desc(kTile, true);
+            constexpr uint64_t kSlot = kTileBytes >> 4;
+            const uint64_t q_desc0 = smem_desc(smem_u32(sm.q[0]), 16);
+            const uint64_t k_desc0 = smem_desc(smem_u32(sm.kv[0]), 16);
+            const uint64_t v_desc0 = smem_desc(smem_u32(sm.kv[0]), kHalfBytes);
+            // S_X = Q_X K_j^T: 16 head-dim elements (32 bytes) per instruction; the second 64-wide half of the
+            // tiles sits 16 KB further.  Called by the elected lane only.
+            auto issue_qk = [&](int x, int j) {
+                const uint64_t kd = k_desc0 + static_cast<uint64_t>((2 * j) % kRing) * kSlot;
+                const uint64_t qd = q_desc0 + static_cast<uint64_t>(x) * kSlot;
+                const uint32_t d_s = tmem + kColS + x * kTile;
+                umma_ss<false>(d_s, qd, kd, idesc_qk);
+                umma_ss<true>(d_s, qd + 2, kd + 2, idesc_qk);
+                umma_ss<true>(d_s, qd + 4, kd + 4, idesc_qk);
+                umma_ss<true>(d_s, qd + 6, kd + 6, idesc_qk);
+                umma_ss<true>(d_s, qd + 1024, kd + 1024, idesc_qk);
+                umma_ss<true>(d_s, qd + 1026, kd + 1026, idesc_qk);
+                umma_ss<true>(d_s, qd + 1028, kd + 1028, idesc_qk);
+                umma_ss<true>(d_s, qd + 1030, kd + 1030, idesc_qk);
+            };
+            // O_X += P_X V_j, keys [64 h, 64 h + 64) of the tile: 16 keys (16 rows of 128 bytes of V, 8 columns of
+            // bf16 pairs of P) per instruction
+            auto issue_pv = [&](int x, int j, int h) {
+                const uint64_t vd = v_desc0 + static_cast<uint64_t>((2 * j + 1) % kRing) * kSlot + h * 512;
+                const uint32_t a_p = tmem + kColS + x * kTile + h * 32, d_o = tmem + kColO + x * kTile;
+                if (j > 0 || h) umma_ts<true>(d_o, a_p, vd, idesc_pv);
+                else umma_ts<false>(d_o, a_p, vd, idesc_pv);
+                umma_ts<true>(d_o, a_p + 8, vd + 128, idesc_pv);
+                umma_ts<true>(d_o, a_p + 16, vd + 256, idesc_pv);
+                umma_ts<true>(d_o, a_p + 24, vd + 384, idesc_pv);
+            };
+            auto wait_bar = [&](uint64_t* bar, uint32_t parity) {
+                return __all_sync(kFull, mbar_wait(smem_u32(bar), parity, abort_flag));
+            };
+            auto wait_unit = [&](int u) { return wait_bar(&sm.kv_full[u % kRing], (u / kRing) & 1); };
+            const int last_x = has_b ? 1 : 0;  // the row tile whose products release the K/V slots
+            bool ok = wait_bar(&sm.q_full[0], 0) && wait_unit(0);
             if (ok) {
                 tc_fence_after();
-                TMEM_LD32(sv, 0, s_addr);
-                TMEM_LD32(sv, 32, s_addr + 32);
-                if (wt == 0) TRACE(half ? 20 : 4);
-                uint32_t vis0 = kFull, vis1 = kFull;
-                bool all_visible = true;
-                if (t_begin < prefix_tiles) {
-                    const int left = P - t_begin * kTile - half * 64;
-                    if (left < 64) {
-                        all_visible = false;
-                        vis0 = left >= 32 ? kFull : (left <= 0 ? 0u : ((1u << left) - 1u));
-                        vis1 = left >= 64 ? kFull : (left <= 32 ? 0u : ((1u << (left - 32)) - 1u));
-                    }
-                } else {
-                    all_visible = false;
-                    const int w0 = (t_begin - prefix_tiles) * 4 + half * 2;
-                    vis0 = w0 < p.W ? mrow[w0] : 0u;
-                    vis1 = w0 + 1 < p.W ? mrow[w0 + 1] : 0u;
-                }
-                tmem_wait_ld();
-                if (!all_visible) { mask32(sv, 0, vis0); mask32(sv, 32, vis1); }
-                float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-#pragma unroll
-                for (int c = 0; c < 64; c += 8)
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        mx4[k] = max3(mx4[k], __uint_as_float(sv[c + 2 * k]), __uint_as_float(sv[c + 2 * k + 1]));
-                m_run = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * p.scale_log2;  // -inf if I see no key of this tile
-                const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
-                float rowsum = 0.f;
-                uint32_t pk[32];
-                exp_block<0, 32>(sv, pk, rowsum, p.scale_log2, m_use);
-                s_ready = 1 < my_tiles && mbar_test(smem_u32(&sm.s_full[1 % kSBufs]), (1 / kSBufs) & 1);
-                exp_block<32, 64>(sv, pk, rowsum, p.scale_log2, m_use);
-                preloaded = __all_sync(kFull, s_ready);
-                if (preloaded) {
+                if (elect_one()) { issue_qk(0, 0); tc_commit(smem_u32(&sm.s_full[0])); if (!has_b) tc_commit(smem_u32(&sm.kv_free[0])); }
+                __syncwarp();
+            }
+            if (ok && has_b) {
+                ok = wait_bar(&sm.q_full[1], 0);
+                if (ok) {
                     tc_fence_after();
-                    const uint32_t s_next = lane_addr + kColS + (1 % kSBufs) * kTile + half * 64;
-                    TMEM_LD32(sv, 0, s_next);
-                    TMEM_LD32(sv, 32, s_next + 32);
+                    if (elect_one()) { issue_qk(1, 0); tc_commit(smem_u32(&sm.s_full[1])); tc_commit(smem_u32(&sm.kv_free[0])); }
+                    __syncwarp();
                 }
-                TMEM_ST32(s_addr, pk, 0);
-                l_run = rowsum;
-                tmem_wait_st();
-                tc_fence_before();
-                mbar_arrive(smem_u32(&sm.p_ready[0][half]));
-                if (wt == 0) TRACE(half ? 21 : 6);
             }
-        }
-        for (int j = 1; j < my_tiles && ok; ++j) {
-            const int t = t_begin + j, b = j % kSBufs;
-            const uint32_t s_addr = lane_addr + kColS + b * kTile + half * 64;
-            [[maybe_unused]] const bool st8 = j == kStampTile;
-            STAMP(st8, 0);
-            STAMP(j == kStampTile + 1, 8);
-            STAMP(j == kStampTile + 2, 9);
-            // Barrier tests, votes and TMEM round trips cost 150-300 cycles each, during which the two
-            // softmax warps of an SM sub-partition (always in the same phase) leave it idle.  So they are
-            // taken off the critical path: the barriers of the coming tile are tested in the middle of
-            // this tile's exponentials, and its scores are requested from TMEM before this tile's P is
-            // stored; the top of the loop normally finds the load in flight.
-            if (!preloaded) {
-                if (!__all_sync(kFull, s_ready)) {
-                    ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.s_full[b]), (j / kSBufs) & 1, abort_flag));
-                    if (!ok) break;  // warp-uniform: the TMEM loads/stores below need the whole warp
-                }
-                tc_fence_after();
-                TMEM_LD32(sv, 0, s_addr);
-                TMEM_LD32(sv, 32, s_addr + 32);
-            }
-            if (wt == 0 && j < 5) TRACE(half ? 20 + 2 * j : 4 + 3 * j);
-            STAMP(st8, 1);
-            bool saw_o_done = j == 0;  // phase j-1 of o_done must be observed exactly once per tile (see below)
-
-            // visibility of this thread's 64 keys
-            uint32_t vis0 = kFull, vis1 = kFull;
-            bool all_visible = true;
-            if (t < prefix_tiles) {
-                const int left = P - t * kTile - half * 64;  // keys of this request in my column range
-                if (left < 64) {
-                    all_visible = false;
-                    vis0 = left >= 32 ? kFull : (left <= 0 ? 0u : ((1u << left) - 1u));
-                    vis1 = left >= 64 ? kFull : (left <= 32 ? 0u : ((1u << (left - 32)) - 1u));
-                }
-            } else {
-                all_visible = false;
-                const int w0 = (t - prefix_tiles) * 4 + half * 2;
-                vis0 = w0 < p.W ? mrow[w0] : 0u;
-                vis1 = w0 + 1 < p.W ? mrow[w0 + 1] : 0u;
-            }
-            tmem_wait_ld();
-            STAMP(st8, 2);
-            if (!all_visible) { mask32(sv, 0, vis0); mask32(sv, 32, vis1); }
-            // Optimistic pass: exponentials relative to the reference maximum as it stands.  P keeps its
-            // relative precision whatever the reference (bf16 has the exponent range of fp32), so the
-            // reference only has to keep the sums away from overflow: it is revisited when a row sum
-            // exceeds 2^24 (or is not finite), and on the first tile, where there is none yet.
-            float rowsum = 0.f;
-            uint32_t pk[32];
-            {
-                const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
-                exp_block<0, 32>(sv, pk, rowsum, p.scale_log2, m_use);
-                // early tests of the coming tile's barriers (results are consumed further down)
-                s_ready = j + 1 < my_tiles && mbar_test(smem_u32(&sm.s_full[(j + 1) % kSBufs]), ((j + 1) / kSBufs) & 1);
-                if (!saw_o_done) saw_o_done = mbar_test(smem_u32(&sm.o_done[half]), (j - 1) & 1);
-                exp_block<32, 64>(sv, pk, rowsum, p.scale_log2, m_use);
-            }
-            STAMP(st8, 3);
-            const bool revisit = m_run == -CUDART_INF_F || !(rowsum < 16777216.f);
-            if (__any_sync(kFull, revisit)) {
-                // exact maximum of my 64 scores; the reference moves only when the maximum outgrew it by 2^8
-                float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-#pragma unroll
-                for (int c = 0; c < 64; c += 8)
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        mx4[k] = max3(mx4[k], __uint_as_float(sv[c + 2 * k]), __uint_as_float(sv[c + 2 * k + 1]));
-                const float m_tile = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * p.scale_log2;
-                const bool bump = m_tile > m_run + 8.f;
-                const float alpha = bump ? ex2(m_run - m_tile) : 1.f;
-                if (bump) { l_run *= alpha; m_run = m_tile; }
-                if (j > 0 && __any_sync(kFull, bump)) {  // O_half holds the sum over the earlier tiles: rescale my row
-                    if (!__all_sync(kFull, saw_o_done)) {
-                        ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[half]), (j - 1) & 1, abort_flag));
+            for (int j = 0; j < my_tiles && ok; ++j) {
+                const bool more = j + 1 < my_tiles;
+                const int uv = 2 * j + 1, sv_slot = uv % kRing;
+                for (int x = 0; x <= last_x && ok; ++x) {
+                    if (x == 0) {
+                        // V_j staged and passed on by the clean-up warp (a slot holds K and V tiles in turn: every
+                        // other use is a V tile), K_{j+1} staged: copies run far ahead, these rarely wait
+                        ok = wait_bar(&sm.v_fix[sv_slot], ((uv / kRing) >> 1) & 1) && (!more || wait_unit(uv + 1));
                         if (!ok) break;
                     }
-                    saw_o_done = true;
+                    // the probabilities arrive in two halves of 64 keys: the product over the first half runs
+                    // while the row tile's threads still exponentiate the second
+                    ok = wait_bar(&sm.p_half[x], j & 1);
+                    if (!ok) break;
                     tc_fence_after();
-#pragma unroll
-                    for (int c0 = 0; c0 < 128; c0 += 32) {
-                        uint32_t ov[32];
-                        TMEM_LD32(ov, 0, o_addr + c0);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * alpha);
-                        TMEM_ST32(o_addr + c0, ov, 0);
+                    if (elect_one()) {
+                        issue_pv(x, j, 0);
+                        tc_commit(smem_u32(&sm.o_half[x]));
                     }
+                    __syncwarp();
+                    ok = wait_bar(&sm.p_ready[x], j & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (elect_one()) {
+                        issue_pv(x, j, 1);
+                        if (x == last_x) tc_commit(smem_u32(&sm.kv_free[sv_slot]));
+                        if (more) {
+                            issue_qk(x, j + 1);
+                            tc_commit(smem_u32(&sm.s_full[x]));
+                            if (x == last_x) tc_commit(smem_u32(&sm.kv_free[(uv + 1) % kRing]));
+                        } else {
+                            tc_commit(smem_u32(&sm.o_final[x]));
+                        }
+                    }
+                    __syncwarp();
                 }
-                const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
-                rowsum = 0.f;
-                exp_block<0, 64>(sv, pk, rowsum, p.scale_log2, m_use);
             }
-            STAMP(st8, 4);
-            // the scores are consumed: request the coming tile's (other S buffer) before storing P
-            preloaded = __all_sync(kFull, s_ready);
-            if (preloaded) {
+        }
+    } else {
+        regs_inc<kRegsSoftmax>();
+        // ---- softmax: thread `row` of group X owns row `row` of row tile rt0 + X: all 128 scores of every KV
+        //      tile, its own reference maximum and sum; nobody else ever touches that row ----
+        const int x = warp >> 2, row = tid & (kTile - 1);
+        if (x == 0 || has_b) {
+            const int grow = (rt0 + x) * kTile + row;   // row among this KV head's rows
+            const int node = grow / p.G;
+            const bool valid = node < n;
+            const uint32_t* mrow = p.anc_mask + (static_cast<size_t>(r) * p.N + (valid ? node : 0)) * p.W;
+            const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+            const uint32_t s_addr = lane_addr + kColS + x * kTile;
+            const uint32_t o_addr = lane_addr + kColO + x * kTile;
+            float m_run = -CUDART_INF_F, l_run = 0.f;  // reference maximum (scaled log2 units; -inf: no key seen yet), sum
+            bool ok = true;
+            // A tile's scores come from tensor memory one half (64 columns) at a time: few registers are live (with
+            // all 128 scores of a row in registers the compiler has no room to keep exponentials in flight), and
+            // there are only two round trips per tile (a load in flight holds the warp back; the other row tile's
+            // warp on the same sub-partition fills the gap).
+            uint32_t sc[64], pk[32];
+            // Per half (64 keys) of a tile, an optimistic pass: exponentials relative to the reference maximum as it
+            // stands.  P keeps its relative precision whatever the reference (bf16 has the exponent range of fp32),
+            // so the reference only has to keep the sums away from overflow: it is revisited when a row sum exceeds
+            // 2^24 (or is not finite), and for a row that sees its first key.  Then the probabilities go over the
+            // scores' own columns and the MMA warp is told.
+            for (int j = 0; j < my_tiles && ok; ++j) {
+                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.s_full[x]), j & 1, abort_flag));
+                if (!ok) break;  // warp-uniform: the TMEM loads/stores below need the whole warp
                 tc_fence_after();
-                const uint32_t s_next = lane_addr + kColS + ((j + 1) % kSBufs) * kTile + half * 64;
-                TMEM_LD32(sv, 0, s_next);
-                TMEM_LD32(sv, 32, s_next + 32);
+                uint32_t vis[4];
+                const bool all_visible = tile_visibility(vis, t_begin + j, prefix_tiles, P, p.W, valid, mrow);
+                // the two halves run through the same code (one copy of the unrolled exponent loop: short CTAs
+                // pay for every instruction they fetch for the first time)
+#pragma unroll 1
+                for (int kh = 0; kh < 2; ++kh) {
+                    tmem_ld64(sc, s_addr + 64 * kh);
+                    const uint32_t vis0 = kh ? vis[2] : vis[0], vis1 = kh ? vis[3] : vis[1];
+                    const bool sees = all_visible || (vis0 | vis1) != 0u;
+                    tmem_wait_ld();
+                    if (!all_visible) { mask32(sc, 0, vis0); mask32(sc, 32, vis1); }
+                    float rowsum = exp_pack_64(sc, pk, p.scale_log2, m_run == -CUDART_INF_F ? 0.f : m_run);
+                    const bool revisit = m_run == -CUDART_INF_F ? sees : !(rowsum < 16777216.f);
+                    if (__any_sync(kFull, revisit)) {
+                        // exact maximum of my 64 scores (still in registers); the reference moves only when the
+                        // maximum outgrew it by 2^8
+                        const float m_tile = max_64(sc) * p.scale_log2;  // -inf if I see no key of this half
+                        const bool bump = m_tile > m_run + 8.f;
+                        const float alpha = bump ? ex2(m_run - m_tile) : 1.f;
+                        if (bump) { l_run *= alpha; m_run = m_tile; }
+                        if ((j > 0 || kh) && __any_sync(kFull, bump)) {
+                            // O_X holds the sum over everything before this half.  The product of tile j-1 completed
+                            // before this tile's scores were announced; the product over this tile's first half is
+                            // waited for here.  Then my row is rescaled.
+                            if (kh && !__all_sync(kFull, mbar_wait(smem_u32(&sm.o_half[x]), j & 1, abort_flag))) { ok = false; break; }
+                            tc_fence_after();
+#pragma unroll 1
+                            for (int c0 = 0; c0 < 128; c0 += 32) {
+                                TMEM_LD32(pk, 0, o_addr + c0);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) pk[c] = __float_as_uint(__uint_as_float(pk[c]) * alpha);
+                                TMEM_ST32(o_addr + c0, pk, 0);
+                            }
+                            tmem_wait_st();
+                        }
+                        rowsum = exp_pack_64(sc, pk, p.scale_log2, m_run == -CUDART_INF_F ? 0.f : m_run);
+                    }
+                    TMEM_ST32(s_addr + 32 * kh, pk, 0);
+                    l_run += rowsum;
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(kh ? &sm.p_ready[x] : &sm.p_half[x]));
+                }
             }
-            TMEM_ST32(s_addr, pk, 0);
-            l_run += rowsum;
-            tmem_wait_st();
-            STAMP(st8, 5);
-            // A parity wait cannot tell phase j-1 from phase j-3: a thread that skipped phases could
-            // sail through a later wait while the product it needs is still running.  So every tile
-            // observes the previous tile's o_done, here at the latest (by now it has long completed).
-            if (!__all_sync(kFull, saw_o_done)) {
-                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[half]), (j - 1) & 1, abort_flag));
-                if (!ok) break;
-            }
-            STAMP(st8, 6);
-            tc_fence_before();
-            mbar_arrive(smem_u32(&sm.p_ready[b][half]));
-            STAMP(st8, 7);
-            if (wt == 0 && j < 5) TRACE(half ? 21 + 2 * j : 6 + 3 * j);
-        }
 
-        if (preloaded) tmem_wait_ld();  // only when the loop was left early: no load may outlive the TMEM allocation
-        STAMP(true, 10);
-        // ---- epilogue: merge the two halves and write each row's 16-bit values straight from registers ----
-        for (int h = 0; h < 2 && ok; ++h)
-            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_done[h]), (my_tiles - 1) & 1, abort_flag));
-        if (tid == 0) TRACE(46);
-        STAMP(true, 11);
-        const bool direct = p.splits == 1;
-        if (ok) {
-            tc_fence_after();
-            sm.xm[half][wt] = m_run;
-            sm.xl[half][wt] = l_run;
-            mbar_arrive(smem_u32(&sm.fin));
-            ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.fin), 0, abort_flag));
-        }
-        STAMP(true, 12);
-        float l_row = 0.f, m_row = -CUDART_INF_F;
-        if (ok) {
-            const float m_o = sm.xm[half ^ 1][wt], l_o = sm.xl[half ^ 1][wt];
-            m_row = fmaxf(m_run, m_o);
-            const float a_self = m_run == -CUDART_INF_F ? 0.f : ex2(m_run - m_row);
-            const float a_other = m_o == -CUDART_INF_F ? 0.f : ex2(m_o - m_row);
-            l_row = l_run * a_self + l_o * a_other;
-            const float f = l_row > 0.f ? 1.f / l_row : 0.f;  // rows leave normalised, also as split partials
-            const float f0 = (half == 0 ? a_self : a_other) * f, f1 = (half == 0 ? a_other : a_self) * f;
-            // this thread merges head-dim columns [64*half, 64*half+64) of its row from both accumulators,
-            // rounds them to 16 bits and writes its 128 contiguous bytes itself: to the output (bf16)
-            // when this CTA saw the whole KV range, else to the split partials (fp16: the rows are
-            // averages of V rows, so fp16's 11 bits are finer than the bf16 rounding of the final output).
-            // (An SM stores ~32 bytes per clock whatever the route: staging the rows for coalesced stores
-            // or for one bulk tensor store was measured and takes the same time.)
-            uint16_t* dst16;
-            if (direct) {
-                dst16 = reinterpret_cast<uint16_t*>(p.out) +
-                        ((static_cast<size_t>(r) * p.N + (valid ? node : 0)) * p.Hq + kvh * p.G + grow % p.G) * kTile + half * 64;
-            } else {
-                dst16 = reinterpret_cast<uint16_t*>(p.part_o) + (part_row0 + wt) * kTile + half * 64;
-            }
+            // ---- epilogue: each thread normalises its row and writes its 256 contiguous bytes itself: to the
+            //      output (bf16) when this CTA saw the whole KV range, else to the split partials (fp16: the rows
+            //      are averages of V rows, so fp16's 11 bits are finer than the bf16 rounding of the final output).
+            //      (An SM stores ~32 bytes per clock whatever the route: staging the rows for coalesced stores
+            //      or for one bulk tensor store was measured and takes the same time.) ----
+            if (ok) ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.o_final[x]), 0, abort_flag));
+            if (ok) {
+                tc_fence_after();
+                const bool direct = p.splits == 1;
+                const float f = l_run > 0.f ? 1.f / l_run : 0.f;  // rows leave normalised, also as split partials
+                uint16_t* dst16;
+                if (direct) {
+                    dst16 = reinterpret_cast<uint16_t*>(p.out) +
+                            ((static_cast<size_t>(r) * p.N + (valid ? node : 0)) * p.Hq + kvh * p.G + grow % p.G) * kTile;
+                } else {
+                    dst16 = reinterpret_cast<uint16_t*>(p.part_o) + (part_row0 + x * kTile + row) * kTile;
+                }
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t o0[32], o1[32], w16[16];
-                TMEM_LD32(o0, 0, lane_addr + kColO + half * 64 + c0);
-                TMEM_LD32(o1, 0, lane_addr + kColO + kTile + half * 64 + c0);
-                tmem_wait_ld();
-                STAMP(c0 == 0, 13);
+                for (int c0 = 0; c0 < 128; c0 += 32) {
+                    uint32_t w16[16];
+                    TMEM_LD32(sc, 0, o_addr + c0);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int q = 0; q < 16; ++q) {
-                    const float a = fmaf(__uint_as_float(o1[2 * q]), f1, __uint_as_float(o0[2 * q]) * f0);
-                    const float b = fmaf(__uint_as_float(o1[2 * q + 1]), f1, __uint_as_float(o0[2 * q + 1]) * f0);
-                    if (direct) {
-                        const __nv_bfloat162 t2 = __floats2bfloat162_rn(a, b);
-                        w16[q] = *reinterpret_cast<const uint32_t*>(&t2);
-                    } else {
-                        const __half2 t2 = __floats2half2_rn(a, b);
-                        w16[q] = *reinterpret_cast<const uint32_t*>(&t2);
+                    for (int q = 0; q < 16; ++q) {
+                        const float a = __uint_as_float(sc[2 * q]) * f, b = __uint_as_float(sc[2 * q + 1]) * f;
+                        if (direct) {
+                            const __nv_bfloat162 t2 = __floats2bfloat162_rn(a, b);
+                            w16[q] = *reinterpret_cast<const uint32_t*>(&t2);
+                        } else {
+                            const __half2 t2 = __floats2half2_rn(a, b);
+                            w16[q] = *reinterpret_cast<const uint32_t*>(&t2);
+                        }
+                    }
+                    if (valid) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            *reinterpret_cast<uint4*>(dst16 + c0 + 8 * u) = make_uint4(w16[4 * u], w16[4 * u + 1], w16[4 * u + 2], w16[4 * u + 3]);
                     }
                 }
                 if (valid) {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        *reinterpret_cast<uint4*>(dst16 + c0 + 8 * u) = make_uint4(w16[4 * u], w16[4 * u + 1], w16[4 * u + 2], w16[4 * u + 3]);
-                }
-            }
-            if (half == 0 && valid) {
-                if (direct) {
-                    if (p.lse) p.lse[(static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + grow % p.G] = (m_row + log2f(l_row)) / kLog2e;
-                } else {
-                    p.part_ml[part_row0 + wt] = make_float2(m_row, l_row);
+                    if (direct) {
+                        if (p.lse) p.lse[(static_cast<size_t>(r) * p.N + node) * p.Hq + kvh * p.G + grow % p.G] = (m_run + log2f(l_run)) / kLog2e;
+                    } else {
+                        p.part_ml[part_row0 + x * kTile + row] = make_float2(m_run, l_run);
+                    }
                 }
             }
         }
-        STAMP(true, 14);
-        STAMP_FLUSH(wt == 0, half ? 32 : 16);
-        if (tid == 0) TRACE(47);
     }
 
     // ---- teardown -------------------------------------------------------------------------------
-    if (tid == 0) TRACE(48);
     tc_fence_before();
     __syncthreads();
-    if (tid == 0) TRACE(3);
     if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -1221,11 +1122,10 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         if (warp == kProducerWarp && lane == 0) {
             // a wait gave up: before the CTA exits, wait (bounded) for every copy still in flight
             uint32_t scratch = 0;
-            mbar_wait(smem_u32(&sm.q_full), 0, &scratch);
-            for (int j = max(0, k_issued - kStages); j < k_issued; ++j)
-                mbar_wait(smem_u32(&sm.k_full[j % kStages]), (j / kStages) & 1, &scratch);
-            for (int j = max(0, v_issued - kStages); j < v_issued; ++j)
-                mbar_wait(smem_u32(&sm.v_full[j % kStages]), (j / kStages) & 1, &scratch);
+            mbar_wait(smem_u32(&sm.q_full[0]), 0, &scratch);
+            if (has_b) mbar_wait(smem_u32(&sm.q_full[1]), 0, &scratch);
+            for (int u = max(0, issued - kRing); u < issued; ++u)
+                mbar_wait(smem_u32(&sm.kv_full[u % kRing]), (u / kRing) & 1, &scratch);
             atomicExch(p.status, kErrTimeout);
         }
         __syncthreads();
@@ -1239,12 +1139,15 @@ __global__ void __launch_bounds__(128)
 combine_kernel(const KernelParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_wait();  // the split partials come from the attention kernel launched just before
+    const int nodes = p.N - p.node0;
     const long long task = static_cast<long long>(blockIdx.x) * 4 + warp;
-    if (task >= static_cast<long long>(p.R) * p.N * p.Hq) return;
+    if (task >= static_cast<long long>(p.R) * nodes * p.Hq) return;
     const int h = static_cast<int>(task % p.Hq);
-    const int node = static_cast<int>((task / p.Hq) % p.N);
-    const int r = static_cast<int>(task / (static_cast<long long>(p.Hq) * p.N));
+    const int node = p.node0 + static_cast<int>((task / p.Hq) % nodes);
+    const int r = static_cast<int>(task / (static_cast<long long>(p.Hq) * nodes));
     const int kvh = h / p.G, grow = node * p.G + h % p.G;
+    const int splits = (p.tail && grow >= p.full_tiles * kTile) ? p.tail_splits : p.splits;
+    if (splits == 1) return;  // written by its CTA directly
     const size_t split_stride = static_cast<size_t>(p.R) * p.Hkv * p.rows_pad;
     const size_t row0 = (static_cast<size_t>(r) * p.Hkv + kvh) * p.rows_pad + grow;
     // One round trip to L2 for everything this row needs: the row count of the request, the (max, sum)
@@ -1253,11 +1156,11 @@ combine_kernel(const KernelParams p) {
     const __half* po = p.part_o + row0 * kTile + lane * 4;
     const int n_r = p.n_rows[r];
     float2 ml = make_float2(-CUDART_INF_F, 0.f);
-    if (lane < p.splits) ml = p.part_ml[lane * split_stride + row0];
+    if (lane < splits) ml = p.part_ml[lane * split_stride + row0];
     uint2 raw[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u)
-        raw[u] = u < p.splits ? *reinterpret_cast<const uint2*>(po + u * split_stride * kTile) : make_uint2(0u, 0u);
+        raw[u] = u < splits ? *reinterpret_cast<const uint2*>(po + u * split_stride * kTile) : make_uint2(0u, 0u);
     if (node >= n_r) return;
     float M = ml.y > 0.f ? ml.x : -CUDART_INF_F;
 #pragma unroll
@@ -1278,8 +1181,8 @@ combine_kernel(const KernelParams p) {
     };
 #pragma unroll
     for (int u = 0; u < 8; ++u)
-        if (u < p.splits) add(u, raw[u]);
-    for (int s = 8; s < p.splits; ++s) add(s, *reinterpret_cast<const uint2*>(po + s * split_stride * kTile));
+        if (u < splits) add(u, raw[u]);
+    for (int s = 8; s < splits; ++s) add(s, *reinterpret_cast<const uint2*>(po + s * split_stride * kTile));
     const float inv = 1.f / l;
     const __nv_bfloat162 b0 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv);
     const __nv_bfloat162 b1 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
@@ -1289,6 +1192,22 @@ combine_kernel(const KernelParams p) {
     const size_t o = ((static_cast<size_t>(r) * p.N + node) * p.Hq + h) * kTile;
     *reinterpret_cast<uint2*>(p.out + o + lane * 4) = w2;
     if (p.lse && lane == 0) p.lse[(static_cast<size_t>(r) * p.N + node) * p.Hq + h] = (M + log2f(l)) / kLog2e;
+}
+
+// A wait that nothing can satisfy: one thread initialises a barrier nobody arrives at, polls it `limit`
+// times, gives up and raises the time-out flag in the device status word, exactly as the attention
+// kernel's waits do.  The kernel returns normally.  (Self-test of the reporting path: see
+// ddtree_selftest_wait_timeout.)
+__global__ void wait_timeout_selftest_kernel(uint32_t* status, uint32_t limit) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort;
+    pdl_wait();
+    if (threadIdx.x == 0) {
+        abort = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait_limit(smem_u32(&bar), 0, &abort, limit)) atomicExch(status, kErrTimeout);
+    }
 }
 
 // ---- host side ---------------------------------------------------------------------------------
@@ -1366,49 +1285,56 @@ int get_map(CUtensorMap* out, const void* base, int rank, uint64_t d1, uint64_t 
     return DDTREE_OK;
 }
 
+constexpr int kSMs = 148;
+
 struct Plan {
-    int row_tiles, rows_pad, splits;
-    int tail;  // the last row tile takes the short-tile path
+    int row_tiles, rows_pad;
+    int full_tiles, pairs, tail;
+    int splits, tail_splits, units;
     size_t off_ml, total;
 };
 
+// How the rows and the KV range of a call are spread over CTAs.  A batch that fills the SMs more than once
+// runs unsplit.  Otherwise every CTA is resident at once, and the KV range is split so that the pairs' CTAs
+// (~2800 cycles per KV tile) and the short tile's CTAs (~1250 cycles per tile) finish together.
 Plan make_plan(const AttnArgs& a) {
     Plan pl;
     pl.row_tiles = (a.N * a.G + kTile - 1) / kTile;
     pl.rows_pad = pl.row_tiles * kTile;
-    const int base = a.R * a.Hkv * pl.row_tiles;
+    pl.tail = (a.N * a.G - (pl.row_tiles - 1) * kTile <= kTailRows) ? 1 : 0;
+    pl.full_tiles = pl.row_tiles - pl.tail;
+    pl.pairs = (pl.full_tiles + 1) / 2;
+    const int groups = a.R * a.Hkv;
     const int max_tiles = (a.max_prefix + kTile - 1) / kTile + (a.N + kTile - 1) / kTile;
-    int s = 1;
-    if (base < 148) {
-        s = 148 / base;
-        const int cap = (max_tiles + 1) / 2;  // at least two KV tiles per split
-        if (s > cap) s = cap;
-        if (s > 32) s = 32;  // the combine kernel gives one lane to each split
-        if (s < 1) s = 1;
+    pl.splits = 1;
+    pl.tail_splits = 1;
+    if (groups * (pl.pairs + pl.tail) < kSMs) {
+        const int budget = kSMs / groups;                   // CTAs per (request, KV head)
+        const int s_cap = std::max(1, std::min(32, (max_tiles + 1) / 2));  // at least two KV tiles per split
+        const int t_cap = std::max(1, std::min(32, (max_tiles + 3) / 4));
+        double best = 1e30;
+        for (int s = 1; s <= (pl.pairs ? s_cap : 1); ++s) {
+            for (int t = 1; t <= (pl.tail ? t_cap : 1); ++t) {
+                if (pl.pairs * s + pl.tail * t > budget) break;
+                const double cf = pl.pairs ? 9000.0 + 2800.0 * ((max_tiles + s - 1) / s) + (s > 1 ? 400.0 * s : 0.0) : 0.0;
+                const double ct = pl.tail ? 7000.0 + 1250.0 * ((max_tiles + t - 1) / t) : 0.0;
+                const double cost = std::max(cf, ct) + 1.0 * (pl.pairs * s + pl.tail * t);  // ties: fewer CTAs
+                if (cost < best) { best = cost; pl.splits = s; pl.tail_splits = t; }
+            }
+        }
     }
-    pl.splits = s;
-    // The short-tile path pays off where the SMs work through several CTAs each: its KV tiles cost half
-    // as much.  When all CTAs run at once (a few requests, KV splits) it does not: the data comes straight
-    // from HBM, its tiles are too short to hide that latency behind three-deep rings, and it would
-    // only finish after the full tiles' CTAs.
-    pl.tail = (base >= 148 && a.N * a.G - (pl.row_tiles - 1) * kTile <= kTailRows && kTailRows % a.G == 0) ? 1 : 0;
-    const size_t rows = static_cast<size_t>(s) * a.R * a.Hkv * pl.rows_pad;
+    pl.units = pl.pairs * pl.splits + pl.tail * pl.tail_splits;
+    const int smax = std::max(pl.splits, pl.tail ? pl.tail_splits : 1);
+    const size_t rows = static_cast<size_t>(smax) * a.R * a.Hkv * pl.rows_pad;
     pl.off_ml = (rows * kTile * 2 + 255) / 256 * 256;
     pl.total = pl.off_ml + (rows * 8 + 255) / 256 * 256;
-    if (s == 1) { pl.off_ml = 0; pl.total = 256; }
+    if (smax == 1) { pl.off_ml = 0; pl.total = 256; }
     return pl;
 }
 
 }  // namespace
 
 size_t tree_attention_bf16_workspace(const AttnArgs& a, const int32_t*) { return make_plan(a).total; }
-
-#ifdef DDTREE_TRACE
-extern "C" int ddtree_debug_set_trace(void* device_buffer) {
-    unsigned long long* ptr = static_cast<unsigned long long*>(device_buffer);
-    return cudaMemcpyToSymbol(g_trace, &ptr, sizeof(ptr)) == cudaSuccess ? 0 : 4;
-}
-#endif
 
 int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host, void* ws, size_t, cudaStream_t st) {
     const Plan pl = make_plan(a);
@@ -1435,7 +1361,11 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
     p.status = device_status_word();
     if (!p.status) return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: no device status word");
     p.R = a.R; p.N = a.N; p.W = a.W; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = a.G;
-    p.splits = pl.splits; p.rows_pad = pl.rows_pad;
+    p.rows_pad = pl.rows_pad;
+    p.full_tiles = pl.full_tiles; p.pairs = pl.pairs; p.splits = pl.splits;
+    p.tail = pl.tail; p.tail_splits = pl.tail_splits; p.units = pl.units;
+    // the combine kernel visits every row when the pairs are split, else only the short tile's rows
+    p.node0 = pl.splits > 1 ? 0 : (pl.full_tiles * kTile) / a.G;
     p.scale_log2 = a.scale * kLog2e;
     p.ordered = 0;
     if (cu_prefix_host && a.R > 1 && a.R <= kMaxOrdered) {
@@ -1468,17 +1398,25 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
             if (dev >= 0 && dev < 64) done[dev] = true;
         }
     }
-    dim3 grid(pl.splits, pl.row_tiles * a.Hkv, a.R);
+    const long long ctas = static_cast<long long>(a.R) * a.Hkv * pl.units;
+    if (ctas > 0x7fffffffLL) return fail(DDTREE_ERR_UNSUPPORTED, "ddtree_tree_attention: grid too large");
+    dim3 grid(static_cast<unsigned>(ctas));
     cudaError_t e = pl.tail
         ? launch_pdl(tree_attention_bf16_kernel<true>, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, mqt, p)
         : launch_pdl(tree_attention_bf16_kernel<false>, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, mqt, p);
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: launch: %s", cudaGetErrorString(e));
-    if (pl.splits > 1) {
-        const long long tasks = static_cast<long long>(a.R) * a.N * a.Hq;
+    if (pl.splits > 1 || (pl.tail && pl.tail_splits > 1)) {
+        const long long tasks = static_cast<long long>(a.R) * (a.N - p.node0) * a.Hq;
         e = launch_pdl(combine_kernel, dim3(static_cast<unsigned>((tasks + 3) / 4)), dim3(128), 0, st, p);
         if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: combine: %s", cudaGetErrorString(e));
     }
     return DDTREE_OK;
+}
+
+cudaError_t launch_wait_timeout_selftest(uint32_t limit, cudaStream_t st) {
+    uint32_t* status = device_status_word();
+    if (!status) return cudaErrorUnknown;
+    return launch_pdl(wait_timeout_selftest_kernel, dim3(1), dim3(32), 0, st, status, limit);
 }
 
 }  // namespace ddtree

@@ -87,14 +87,6 @@ __device__ __forceinline__ double warp_sum(double x) {
     return x;
 }
 
-#ifdef DDTREE_TRACE
-__device__ long long* g_build_trace = nullptr;
-#define BTRACE(idx) do { if (g_build_trace && blockIdx.x == 0 && threadIdx.x == 0) { long long t_; \
-    asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_) :: "memory"); g_build_trace[idx] = t_; } } while (0)
-#else
-#define BTRACE(idx) ((void)0)
-#endif
-
 struct Shared {
     float logq[kMaxL * kMaxK];
     int tok[kMaxL * kMaxK];
@@ -133,7 +125,6 @@ tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restric
     const int N = B + 1, W = (N + 31) / 32;
 
     pdl_wait();
-    BTRACE(0);
     // ---- 1. merge chunk partials: one warp per draft position ---------------------------------
     for (int i = warp; i < L; i += kWarps) {
         const size_t row = static_cast<size_t>(r) * L + i;
@@ -240,9 +231,7 @@ tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restric
         }
     }
     if (tid < kMaxL + 2) { sh.lvl_cnt[tid] = 0; sh.lvl_cur[tid] = 0; }
-    BTRACE(1);
     __syncthreads();
-    BTRACE(2);
 
     // ---- 2. best-first selection (Algorithm 1) on warp 0 ---------------------------------------
     if (warp == 0) {
@@ -255,21 +244,13 @@ tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restric
         int bests = lane == 0 ? 0 : -1;
         const unsigned none = orderable(-CUDART_INF_F);
         __syncwarp();
-#ifdef DDTREE_TRACE
-        long long ps[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#define PSTAMP(i) do { if (t == 20) { long long t_; asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_)); ps[i] = t_; } } while (0)
-#else
-#define PSTAMP(i) ((void)0)
-#endif
         for (int t = 0; t < B; ++t) {
-            PSTAMP(0);
             const unsigned key = orderable(bestv);
             const unsigned mx = __reduce_max_sync(kFull, key);
             if (mx == none) break;  // heap empty: fewer than B prefixes exist in S_K
             const int src = __ffs(__ballot_sync(kFull, key == mx)) - 1;
             const int u = __shfl_sync(kFull, bests, src);
             const float v = from_orderable(mx);  // the winning candidate's score
-            PSTAMP(1);
             const int du = sh.depth[u], cu = sh.cc[u];
             const float su = sh.sigma[u];
             const int n = count++;
@@ -295,17 +276,16 @@ tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restric
 #pragma unroll 4
                 for (int i = 0; i < trips; ++i) look(i);
             }
-            PSTAMP(2);
             const float cand_u = (cu + 1 < K) ? su + sh.logq[du * K + cu + 1] : -CUDART_INF_F;
             const float cand_n = (du + 1 < L) ? v + sh.logq[(du + 1) * K] : -CUDART_INF_F;
-            // ties go to the lowest slot, as in a scan over the slots in ascending order
+            // within a lane equal scores go to the lower slot; across lanes the pop takes the lowest lane (any
+            // order of equal scores is a valid pop order: the contract is the node set)
             const bool take_u = (lane == (u & 31)) & ((cand_u > bestv) | ((cand_u == bestv) & (u < bests)));
             bestv = take_u ? cand_u : bestv;
             bests = take_u ? u : bests;
             const bool take_n = (lane == (n & 31)) & (cand_n > bestv);
             bestv = take_n ? cand_n : bestv;
             bests = take_n ? n : bests;
-            PSTAMP(3);
             __syncwarp();  // all lanes have read u's state and their slots before lane 0 overwrites them
             {   // lane 0 writes; the other lanes store the same values to a spare slot instead of branching
                 const int wn = lane == 0 ? n : kSlots - 1, wu = lane == 0 ? u : kSlots - 1;
@@ -319,13 +299,8 @@ tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restric
                 sh.cand[wu] = cand_u;
             }
             __syncwarp();
-            PSTAMP(4);
         }
         __syncwarp();
-        BTRACE(3);
-#ifdef DDTREE_TRACE
-        if (g_build_trace && blockIdx.x == 0 && lane == 0) for (int i = 0; i < 5; ++i) g_build_trace[8 + i] = ps[i];
-#endif
 
         // ---- 3. level order: rows sorted by (depth, parent row, rank) --------------------------
         for (int j = lane; j < count; j += 32) atomicAdd(&sh.lvl_cnt[sh.depth[j]], 1);
@@ -372,7 +347,6 @@ tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restric
             __syncwarp();
         }
     }
-    BTRACE(4);
     __syncthreads();
 
     // ---- 4. write the verifier's inputs --------------------------------------------------------
@@ -416,17 +390,9 @@ tree_build_kernel(int L, int V, int K, int B, int chunks, const float* __restric
         }
         anc_mask[o * W + idx] = bits;
     }
-    BTRACE(5);
 }
 
 }  // namespace
-
-#ifdef DDTREE_TRACE
-extern "C" int ddtree_debug_set_build_trace(void* device_buffer) {
-    long long* ptr = static_cast<long long*>(device_buffer);
-    return cudaMemcpyToSymbol(g_build_trace, &ptr, sizeof(ptr)) == cudaSuccess ? 0 : 4;
-}
-#endif
 
 cudaError_t launch_tree_build(int R, int L, int V, int K, int B, const BuildPartialLayout& lay, const void* ws,
                               const void* logits, int dt, int64_t row_stride,

@@ -58,3 +58,51 @@ def tree_arrays_equal(ct: orc.CompiledTree, tree, r: int) -> None:
     got_mask = tree.anc_mask[r].cpu().numpy().view(np.uint32)
     np.testing.assert_array_equal(got_mask, ct.mask, err_msg="anc_mask")
     np.testing.assert_allclose(tree.node_logprob[r].cpu().numpy(), ct.logprob, atol=2e-4, rtol=0)
+
+
+class Guard:
+    """CUDA tensors between two poisoned margins.  The GPU tests hand every output and workspace of a call
+    to the library in such a tensor and check afterwards that the margins still hold the poison: a kernel
+    that writes outside the buffer it was given is caught without a memory checker."""
+
+    MARGIN = 4096  # bytes on either side (keeps the 256-byte alignment of the payload)
+    POISON = 0xA5
+
+    def __init__(self):
+        self.items = []
+
+    def empty(self, shape, dtype, fill=None):
+        import torch
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        buf = torch.full((2 * self.MARGIN + (n + 255) // 256 * 256,), self.POISON, dtype=torch.uint8, device="cuda")
+        view = buf[self.MARGIN:self.MARGIN + n].view(dtype).view(*shape)
+        if fill is not None:
+            view.fill_(fill)
+        self.items.append((buf, n))
+        return view
+
+    def check(self):
+        import torch
+        torch.cuda.synchronize()
+        for k, (buf, n) in enumerate(self.items):
+            assert bool((buf[:self.MARGIN] == self.POISON).all()), f"buffer {k}: bytes before it were overwritten"
+            assert bool((buf[self.MARGIN + n:] == self.POISON).all()), f"buffer {k}: bytes behind it were overwritten"
+
+
+def guarded_tree(g: Guard, R: int, L: int, K: int, B: int):
+    """A Tree (outputs of ddtree_build) whose every array sits between guard bands."""
+    import torch
+    import paper_2604_12989_b200 as dd
+    N, W = B + 1, (B + 1 + 31) // 32
+    i32, f32 = torch.int32, torch.float32
+    return dd.Tree(g.empty((R,), i32), g.empty((R, N), i32), g.empty((R, N), i32), g.empty((R, N), i32),
+                   g.empty((R, N), i32), g.empty((R, N, W), i32), g.empty((R, N), i32), g.empty((R, N), i32),
+                   g.empty((R, N), f32), g.empty((R, L, K), i32), g.empty((R, L, K), f32), B, L, K)
+
+
+def guarded_acceptance(g: Guard, R: int, L: int, N: int):
+    import torch
+    import paper_2604_12989_b200 as dd
+    i32 = torch.int32
+    return dd.Acceptance(g.empty((R,), i32), g.empty((R, L), i32), g.empty((R, L), i32), g.empty((R,), i32),
+                         g.empty((R, N), i32))

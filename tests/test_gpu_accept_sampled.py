@@ -30,8 +30,11 @@ def run_and_compare(w, trees, tl, T, ks):
     par = torch.from_numpy(np.stack([tr.parent for tr in trees])).cuda()
     n_rows = torch.tensor([tr.n_rows for tr in trees], dtype=torch.int32).cuda()
     u = torch.from_numpy(ks.astype(np.uint32).view(np.int32)).cuda()
-    acc = dd.ddtree_accept_sampled(t, w.L, tok, par, n_rows, T, u)
-    torch.cuda.synchronize()
+    g = cases.Guard()
+    ws = g.empty((max(256, dd.lib().ddtree_accept_sampled_workspace_bytes(w.R, w.B, w.V)),), torch.uint8)
+    acc = dd.ddtree_accept_sampled(t, w.L, tok, par, n_rows, T, u, workspace=ws,
+                                   out=cases.guarded_acceptance(g, w.R, w.L, w.N))
+    g.check()
     lens = []
     for r in range(w.R):
         n = trees[r].n_rows
@@ -146,3 +149,95 @@ def test_random_shapes(seed):
     tl = np.stack([wl.target_logits(w, trees[r].depth, r, "peak") for r in range(w.R)])
     ks = rng.integers(0, 2 ** 32, (w.R, w.N), dtype=np.uint64)
     run_and_compare(w, trees, tl, T, ks)
+
+
+# ---------------------------------------------------------------------------------------------
+# The kernel against the rule itself (Section 4.4: the target's choice is a sample from its
+# distribution at temperature T), not against the oracle's operation list: an inverse-CDF draw over
+# the exact softmax, written out here in float64.
+# ---------------------------------------------------------------------------------------------
+
+def exact_inverse_cdf(x64, T, ks):
+    """For every row: p = softmax(x / T) in float64, u = k / 2^32, the smallest v with cdf(v) > u, and the
+    distance from u to the nearest cdf step on either side of that token (how close the draw was)."""
+    z = x64 / T
+    z = z - z.max(axis=1, keepdims=True)
+    p = np.exp(z)
+    p /= p.sum(axis=1, keepdims=True)
+    cdf = np.cumsum(p, axis=1)
+    u = ks.astype(np.float64) / 2.0 ** 32
+    choice = np.array([int(np.searchsorted(cdf[i], u[i], side="right")) for i in range(x64.shape[0])])
+    choice = np.minimum(choice, x64.shape[1] - 1)
+    hi = cdf[np.arange(len(u)), choice]
+    lo = np.where(choice > 0, cdf[np.arange(len(u)), np.maximum(choice - 1, 0)], 0.0)
+    return choice, np.minimum(np.abs(hi - u), np.abs(u - lo))
+
+
+def drawn_tokens(w, trees, t_dev, T, ks):
+    import paper_2604_12989_b200 as dd
+    tok = torch.from_numpy(np.stack([tr.token for tr in trees])).cuda()
+    par = torch.from_numpy(np.stack([tr.parent for tr in trees])).cuda()
+    n_rows = torch.tensor([tr.n_rows for tr in trees], dtype=torch.int32).cuda()
+    u = torch.from_numpy(ks.astype(np.uint32).view(np.int32)).cuda()
+    acc = dd.ddtree_accept_sampled(t_dev, w.L, tok, par, n_rows, T, u)
+    torch.cuda.synchronize()
+    return acc.node_argmax.cpu().numpy()
+
+
+@pytest.mark.parametrize("T", [0.7, 1.0, 1.5])
+def test_draws_equal_the_exact_inverse_cdf_at_full_vocabulary(T):
+    """Config 1's target logits (65 rows x 151936 bf16 values), as many sets of random inputs per temperature
+    as it takes to compare more than 1000 draws.  Every draw whose u is further than 1e-5 from a step of the exact
+    cdf must give the exact token (the fixed-point weights are within 5e-6 of the exact numerators, so the
+    two cdfs differ by less than that everywhere)."""
+    w = wl.WORKLOADS[1]
+    trees = make_trees(w, "peak")
+    tl = np.stack([wl.target_logits(w, trees[r].depth, r, "peak") for r in range(w.R)])
+    x64 = wl.bf16_to_f64(tl[0])
+    t_dev = aligned_rows(cases.to_torch(tl, True))
+    n = trees[0].n_rows
+    compared = 0
+    for rep in range(96):
+        if compared >= 1000:
+            break
+        ks = np.random.default_rng([int(T * 100), rep]).integers(0, 2 ** 32, (w.R, w.N), dtype=np.uint64)
+        got = drawn_tokens(w, trees, t_dev, T, ks)[0, :n]
+        want, margin = exact_inverse_cdf(x64[:n], T, ks[0, :n])
+        clear = margin >= 1e-5
+        np.testing.assert_array_equal(got[clear], want[clear])
+        compared += int(clear.sum())
+    assert compared >= 1000
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_draw_frequencies_follow_the_softmax(dtype):
+    """Many rows with the same logits and independent random inputs: the empirical token frequencies of the
+    GPU draws match softmax(x / T) within five standard errors, and the draws are the exact inverse-CDF
+    tokens wherever u is clear of a cdf step."""
+    V, T = 48, 1.3
+    w = wl.small_workload(R=8, L=8, V=V, K=4, B=1024, Hq=4, Hkv=2, d=64, dtype=dtype, prefix_lens=tuple([2] * 8), index=74)
+    trees = make_trees(w)
+    rng = np.random.default_rng(74)
+    row = (rng.standard_normal(V) * 2.0).astype(np.float32)
+    row = wl.round_through_bf16(row)  # exactly representable in both dtypes
+    x = np.broadcast_to(row, (w.R, w.N, V)).copy()
+    tl = wl.f32_to_bf16_bits(x) if dtype == "bf16" else x
+    ks = rng.integers(0, 2 ** 32, (w.R, w.N), dtype=np.uint64)
+    got = drawn_tokens(w, trees, aligned_rows(cases.to_torch(tl, dtype == "bf16")), T, ks)
+    draws, wants, margins = [], [], []
+    for r in range(w.R):
+        n = trees[r].n_rows
+        draws.append(got[r, :n])
+        want, margin = exact_inverse_cdf(x[r, :n].astype(np.float64), T, ks[r, :n])
+        wants.append(want)
+        margins.append(margin)
+    draws, wants, margins = np.concatenate(draws), np.concatenate(wants), np.concatenate(margins)
+    assert len(draws) >= 2000
+    clear = margins >= 1e-5
+    np.testing.assert_array_equal(draws[clear], wants[clear])
+    z = row.astype(np.float64) / T
+    p = np.exp(z - z.max())
+    p /= p.sum()
+    freq = np.bincount(draws, minlength=V) / len(draws)
+    se = np.sqrt(p * (1 - p) / len(draws))
+    assert (np.abs(freq - p) <= 5 * se + 1e-4).all(), np.abs(freq - p).max()

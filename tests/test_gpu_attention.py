@@ -19,9 +19,14 @@ def gpu_attention(w, att, trees, with_lse=True):
     n_rows = torch.tensor([t.n_rows for t in trees], dtype=torch.int32).cuda()
     cu = torch.from_numpy(att.cu_prefix).cuda()
     q, kc, vc, kt, vt = (cases.to_torch(getattr(att, n), bf) for n in ("q", "k_cache", "v_cache", "k_tree", "v_tree"))
-    lse = torch.zeros(w.R, w.N, w.Hq, dtype=torch.float32, device="cuda") if with_lse else None
-    out = dd.ddtree_tree_attention(q, kc, vc, att.cu_prefix.tolist(), cu, kt, vt, mask, n_rows, lse=lse)
-    torch.cuda.synchronize()
+    # out, lse and the workspace sit between poisoned guard bands: nothing may be written outside them
+    g = cases.Guard()
+    lse = g.empty((w.R, w.N, w.Hq), torch.float32, fill=0) if with_lse else None
+    out = g.empty(tuple(q.shape), q.dtype, fill=0)
+    ws = g.empty((max(256, dd.tree_attention_workspace_bytes(w.R, w.B, w.Hq, w.Hkv, w.d, 1 if bf else 0,
+                                                             att.cu_prefix.tolist())),), torch.uint8)
+    dd.ddtree_tree_attention(q, kc, vc, att.cu_prefix.tolist(), cu, kt, vt, mask, n_rows, out=out, lse=lse, workspace=ws)
+    g.check()
     dd.device_status()
     return out.float().cpu().numpy().astype(np.float64), (lse.cpu().numpy() if with_lse else None)
 
@@ -337,3 +342,46 @@ def test_bf16_random_shapes(seed):
     compare(w, att, trees, out, lse)
     for r in range(R):
         assert (out[r, trees[r].n_rows:] == 0).all()  # rows past the tree are left alone
+
+
+def test_bf16_padding_inputs_may_hold_nan():
+    """Rows of the inputs that the call must ignore are filled with NaN bit patterns: tree rows >= n_rows of
+    q, k_tree and v_tree (one request's tree is smaller than the budget), and spare cache rows behind the
+    last request's prefix.  Masked probabilities are zero, but the value rows of a masked key still travel
+    through the tensor cores in a 128-key tile, so the kernel has to clear them: every valid row must still
+    match the oracle, on the split path (one request), on the unsplit path (a batch that fills the GPU) and
+    on the short last row tile."""
+    import dataclasses
+    import paper_2604_12989_b200 as dd
+    nan16 = np.uint16(0x7FC0)
+    for R, B, Hq, Hkv, prefix in ((1, 200, 8, 2, (300,)), (2, 70, 8, 2, (127, 5)), (40, 35, 16, 4, None), (75, 35, 4, 1, None)):
+        if prefix is None:
+            prefix = short_tile_prefixes(R, B, 300)
+        w, att, trees = bf16_case(R, B, Hq, Hkv, prefix, seed=B)
+        for r in range(0, R, 2):  # every other request: a smaller tree (the first rows of a level-order tree are a tree)
+            trees[r] = dataclasses.replace(trees[r], n_rows=max(1, trees[r].n_rows - 3 - r % 5))
+        for r in range(R):
+            n = trees[r].n_rows
+            att.q[r, n:] = nan16
+            att.k_tree[r, n:] = nan16
+            att.v_tree[r, n:] = nan16
+        bf = True
+        mask = torch.from_numpy(np.stack([t.mask for t in trees]).view(np.int32)).cuda()
+        n_rows = torch.tensor([t.n_rows for t in trees], dtype=torch.int32).cuda()
+        cu = torch.from_numpy(att.cu_prefix).cuda()
+        q, kc, vc, kt, vt = (cases.to_torch(getattr(att, nm), bf) for nm in ("q", "k_cache", "v_cache", "k_tree", "v_tree"))
+        # spare rows behind the packed cache (what a cache with room for the accepted path looks like)
+        spare = torch.full((64,) + tuple(kc.shape[1:]), float("nan"), dtype=kc.dtype, device="cuda")
+        kc2, vc2 = torch.cat([kc, spare]), torch.cat([vc, spare])
+        total = int(att.cu_prefix[-1])
+        out = torch.zeros_like(q)
+        lse = torch.zeros(w.R, w.N, w.Hq, dtype=torch.float32, device="cuda")
+        dd.ddtree_tree_attention(q, kc2[:total], vc2[:total], att.cu_prefix.tolist(), cu, kt, vt, mask, n_rows, out=out, lse=lse)
+        torch.cuda.synchronize()
+        dd.device_status()
+        got = out.float().cpu().numpy().astype(np.float64)
+        for r in range(R):  # the oracle never looks at rows >= n_rows
+            n = trees[r].n_rows
+            assert np.isfinite(got[r, :n]).all(), f"request {r}: NaN leaked into a valid row"
+            assert (got[r, n:] == 0).all()
+        compare(w, att, trees, got, lse.cpu().numpy())
