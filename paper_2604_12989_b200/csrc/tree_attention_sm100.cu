@@ -886,13 +886,18 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         } else if (warp == kFixWarp) {
             // ---- V clean-up: every staged V tile passes through this warp on its way to the MMA warp; rows
             //      that no row may see are cleared (see clear_v_rows).  The copies run tiles ahead of the
-            //      products, so the relay is off the critical path. ----
-            for (int j = 0; j < my_tiles; ++j) {
-                const int u = 2 * j + 1, s = u % kRing;
+            //      products, so the relay is off the critical path.  The warp watches the arrival of every
+            //      ring unit in order, K tiles included: a parity wait only tells a phase from its neighbour,
+            //      so a waiter that skipped the K tile's phase of a slot could take that phase still being
+            //      open for the completion of the V tile's phase after it. ----
+            for (int u = 0; u < units_total; ++u) {
+                const int s = u % kRing;
                 if (!__all_sync(kFull, mbar_wait(smem_u32(&sm.kv_full[s]), (u / kRing) & 1, abort_flag))) break;
-                const int first = keys_in_tile(t_begin + j, prefix_tiles, P, n);
-                if (first < kTile) clear_v_rows(sm.kv[s], first, lane);
-                if (lane == 0) mbar_arrive(smem_u32(&sm.v_fix[s]));
+                if (u & 1) {
+                    const int first = keys_in_tile(t_begin + (u >> 1), prefix_tiles, P, n);
+                    if (first < kTile) clear_v_rows(sm.kv[s], first, lane);
+                    if (lane == 0) mbar_arrive(smem_u32(&sm.v_fix[s]));
+                }
             }
         } else if (warp == kMmaWarp) {
             // ---- MMA issuer: the whole warp walks the loop (so that addresses live in uniform registers)

@@ -385,3 +385,40 @@ def test_bf16_padding_inputs_may_hold_nan():
             assert np.isfinite(got[r, :n]).all(), f"request {r}: NaN leaked into a valid row"
             assert (got[r, n:] == 0).all()
         compare(w, att, trees, got, lse.cpu().numpy())
+
+
+def test_bf16_long_trains_of_launches_stay_identical():
+    """Hundreds of back-to-back launches on the large-budget workload's shapes, rotating over input sets larger
+    than L2 so that the copies' arrival order varies: every launch must give bit for bit what the first launch
+    on the same inputs gave, and no device-side wait may give up.  (A warp that watched only every other phase
+    of a copy barrier once passed a wait early when a K tile landed after the V tile behind it: a rare
+    timing, seen only in long trains.)"""
+    import paper_2604_12989_b200 as dd
+    w = wl.WORKLOADS[2]
+    att, trees = make_case(w, "lit")
+    mask = torch.from_numpy(np.stack([t.mask for t in trees]).view(np.int32)).cuda()
+    n_rows = torch.tensor([t.n_rows for t in trees], dtype=torch.int32).cuda()
+    cu = torch.from_numpy(att.cu_prefix).cuda()
+    base = [cases.to_torch(getattr(att, n), True) for n in ("q", "k_cache", "v_cache", "k_tree", "v_tree")]
+    sets = [base] + [[torch.randn_like(t, dtype=torch.float32).to(torch.bfloat16) for t in base] for _ in range(2)]
+    ws = torch.empty(max(256, dd.tree_attention_workspace_bytes(w.R, w.B, w.Hq, w.Hkv, w.d, 1, att.cu_prefix.tolist())),
+                     dtype=torch.uint8, device="cuda")
+    outs = [torch.zeros_like(base[0]) for _ in sets]
+    first = []
+    for k, (q, kc, vc, kt, vt) in enumerate(sets):
+        dd.ddtree_tree_attention(q, kc, vc, att.cu_prefix.tolist(), cu, kt, vt, mask, n_rows, out=outs[k], workspace=ws)
+        first.append(outs[k].clone())
+    torch.cuda.synchronize()
+    dd.device_status()
+    for it in range(600):
+        k = it % len(sets)
+        q, kc, vc, kt, vt = sets[k]
+        dd.ddtree_tree_attention(q, kc, vc, att.cu_prefix.tolist(), cu, kt, vt, mask, n_rows, out=outs[k], workspace=ws)
+        if it % 100 == 99:
+            torch.cuda.synchronize()
+            for a, b in zip(outs, first):
+                assert torch.equal(a, b), f"launch {it}: output changed"
+    torch.cuda.synchronize()
+    dd.device_status()
+    out0 = first[0].float().cpu().numpy().astype(np.float64)
+    compare(w, att, trees, out0, None, sampled_pairs(w, trees, (), 24, 2))
