@@ -59,8 +59,8 @@ const char* ddtree_status_string(int status);
 const char* ddtree_last_error(void);
 
 /* ------------------------------------------------------------------------------------------
- * ddtree_build -- Sections 3, 4.3 (Algorithm 1) and 4.4 ("flatten ... position ids ... tree
- * attention" inputs).
+ * ddtree_build -- Sections 3, 4.3 (Algorithm 1) and 4.4 (the verifier's inputs: the tree as one
+ * sequence, position ids, the attention mask).
  *
  * For every request r and draft position i = 1..L, reads the logit row l_i (row r*L + i-1 of
  * `drafter_logits`, V elements of type `dt`, rows `row_stride_elems` apart), forms
@@ -122,10 +122,16 @@ int ddtree_build(const void* drafter_logits, int dt, int64_t row_stride_elems,
  *   out              [R, B+1, Hq, d]      same element type as q; rows >= n_rows[r] are left untouched
  *   lse_or_null      [R, B+1, Hq] fp32    optional natural-log sum of exp(scaled scores)
  * dt = DDTREE_BF16: bf16 inputs, fp32 accumulation on the tensor cores, probabilities rounded to
- *   bf16 before the PV product (when the KV range of a request is split over several CTAs, each
- *   part's normalised rows pass through fp16 before they are merged); requires d == 128.  dt = DDTREE_F32: fp32 FMA arithmetic; d in
- *   {64, 128}.  Hq must be a multiple of Hkv with Hq/Hkv in {1, 2, 4, 8, 16}.
- * softmax_scale 0 means 1/sqrt(d).  All tensors must be 16-byte aligned.
+ *   bf16 before the PV product; requires d == 128.  When the KV range of a request is split over
+ *   several CTAs (batches that do not fill the GPU), each part's normalised rows pass through fp16 before
+ *   they are merged: the values must then stay below fp16's largest finite value, |v| < 65504 (an output
+ *   row is a convex combination of V rows).  dt = DDTREE_F32: fp32 FMA arithmetic; d in {64, 128}.
+ *   Hq must be a multiple of Hkv with Hq/Hkv in {1, 2, 4, 8, 16}.
+ * Rows the call must ignore may hold anything, NaN and Inf bit patterns included: rows >= n_rows[r] of q,
+ *   k_tree and v_tree, and memory behind the packed cache.  (A masked key's probability is zero, but its
+ *   value row still travels through the tensor cores in a 128-key tile; the kernel clears such rows first.)
+ *   Visible keys and values must be finite.
+ * softmax_scale 0 means 1/sqrt(d); it must be positive.  All tensors must be 16-byte aligned.
  * workspace: at least ddtree_tree_attention_workspace_bytes(...) bytes, 16-byte aligned.
  * ------------------------------------------------------------------------------------------ */
 size_t ddtree_tree_attention_workspace_bytes(int R, int B, int Hq, int Hkv, int d, int dt,
@@ -168,10 +174,10 @@ int ddtree_accept(const void* target_logits, int dt, int64_t row_stride_elems,
                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
- * ddtree_accept_sampled -- Section 4.4 (verifier walk under the temperature-based decoding rule:
- * "verification follows the target model's own decoding rule, whether greedy or temperature-based
- * sampling").  The walk is that of ddtree_accept; the target's choice at a row is a draw from
- * softmax(target_logits[row] / temperature) instead of the arg-max.
+ * ddtree_accept_sampled -- Section 4.4 (verifier walk when the target decodes by sampling at a
+ * temperature instead of greedily; the paper lets the verification use either rule).  The walk is that of
+ * ddtree_accept; the target's choice at a row is a draw from softmax(target_logits[row] / temperature)
+ * instead of the arg-max.
  *
  * The paper does not say how the draw is made.  Here it is a function of the row, the temperature and
  * one caller-supplied 32-bit integer per row, defined on integers so that it does not depend on the
@@ -207,9 +213,10 @@ int ddtree_accept_sampled(const void* target_logits, int dt, int64_t row_stride_
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
- * ddtree_rope_tree -- Section 4.4: "we assign position ids by tree depth so that the verifier applies the
- * correct positional encoding".  Applies the rotary positional encoding (half-split form, as the paper's
- * Qwen3 targets use) to the tree's query and key rows IN PLACE, at the position ids ddtree_build wrote:
+ * ddtree_rope_tree -- Section 4.4 (position ids follow the tree depth, so that the verifier encodes every
+ * node at the position it would have in its own branch).  Applies the rotary positional encoding (half-split
+ * form, as the paper's Qwen3 targets use) to the tree's query and key rows IN PLACE, at the position ids
+ * ddtree_build wrote:
  * for every valid row i, every head and every j < d/2, with a = position_ids[r, i] * rope_theta^(-2j/d),
  *     (x[j], x[j + d/2])  <-  (x[j] cos a - x[j + d/2] sin a,  x[j + d/2] cos a + x[j] sin a).
  * Angles are evaluated in double precision, the rotation in float32, results rounded to dt.

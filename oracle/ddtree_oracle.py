@@ -243,7 +243,7 @@ def tree_attention(q: np.ndarray, k_prefix: np.ndarray, v_prefix: np.ndarray, k_
 
 def node_argmax(target_logits: np.ndarray) -> np.ndarray:
     """The target's greedy choice at every row: the smallest token id attaining the
-    row maximum (Section 4.4, "the target model's own decoding rule", greedy)."""
+    row maximum (Section 4.4: the target's own decoding rule, greedy case)."""
     x = np.asarray(target_logits, np.float64)
     return np.argmax(x, axis=-1).astype(np.int32)  # numpy returns the first maximum
 
@@ -281,8 +281,8 @@ def accept_walk(token: np.ndarray, parent: np.ndarray, n_rows: int, choice: np.n
 # Section 4.4: verification walk (temperature-based sampling rule)
 # --------------------------------------------------------------------------
 #
-# "Verification then follows the target model's own decoding rule, whether greedy
-# or temperature-based sampling": at temperature T > 0 the target's choice at a
+# Section 4.4 lets the verification follow whichever rule the target decodes by,
+# greedy or sampling at a temperature: at temperature T > 0 the target's choice at a
 # row is a token drawn from softmax(t / T).  The paper does not say how the draw
 # is made.  For the draw to be a function of its inputs that two programs can
 # agree on bit for bit, it is defined here as an inverse-CDF draw in token order
@@ -360,8 +360,8 @@ def node_sampled(target_logits: np.ndarray, temperature: float, uniforms: np.nda
 
 def rope(x: np.ndarray, positions: np.ndarray, theta: float) -> np.ndarray:
     """Rotary positional encoding of the rows of x ([rows, heads, d], d even) at the given integer
-    positions ("we assign position ids by tree depth so that the verifier applies the correct positional
-    encoding", Section 4.4; the target models of the paper, Qwen3, use rotary embeddings in the
+    positions (Section 4.4 assigns position ids by tree depth so that every node is encoded at the position
+    it would have in its own branch; the target models of the paper, Qwen3, use rotary embeddings in the
     half-split form).  Pair (j, j + d/2) of every head is rotated by the angle
     positions[row] * theta^(-2j/d): as complex numbers z_j = x_j + i x_{j+d/2}, out = z_j * exp(i * angle)."""
     x = np.asarray(x, np.float64)

@@ -103,6 +103,17 @@ def _stream(stream=None) -> int:
     return (stream or torch.cuda.current_stream()).cuda_stream
 
 
+def _scratch(nbytes: int, device, stream=None):
+    """A temporary workspace for one call.  The kernels are only enqueued when the call returns, so the block
+    must not go back to the caching allocator's pool of another stream while they run: when the call is made on a
+    stream that is not the current one, the block is tied to that stream."""
+    import torch
+    t = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    if stream is not None and stream != torch.cuda.current_stream(device):
+        t.record_stream(stream)
+    return t
+
+
 @dataclass
 class Tree:
     """Outputs of ddtree_build (torch CUDA tensors).  Shapes: [R] or [R, B+1(, W)]."""
@@ -139,7 +150,7 @@ def ddtree_build(drafter_logits, K: int, B: int, root_token, prefix_len, workspa
                    torch.empty(R, L, K, **i32), torch.empty(R, L, K, dtype=torch.float32, device=dev), B, L, K)
     need = lib().ddtree_build_workspace_bytes(R, L, V, K, B)
     if workspace is None:
-        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        workspace = _scratch(need, dev, stream)
     _check(lib().ddtree_build(
         drafter_logits.data_ptr(), _dtype_code(drafter_logits), drafter_logits.stride(1), R, L, V, K, B,
         root_token.data_ptr(), prefix_len.data_ptr(), out.n_rows.data_ptr(), out.node_token.data_ptr(),
@@ -171,7 +182,7 @@ def ddtree_tree_attention(q, k_cache, v_cache, cu_prefix_host, cu_prefix, k_tree
     arr = (ctypes.c_int32 * (R + 1))(*[int(x) for x in cu_prefix_host])
     if workspace is None:
         need = lib().ddtree_tree_attention_workspace_bytes(R, B, Hq, Hkv, d, code, ctypes.addressof(arr))
-        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=q.device)
+        workspace = _scratch(need, q.device, stream)
     _check(lib().ddtree_tree_attention(
         q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), ctypes.addressof(arr), cu_prefix.data_ptr(),
         k_tree.data_ptr(), v_tree.data_ptr(), anc_mask.data_ptr(), n_rows.data_ptr(), out.data_ptr(), _ptr(lse),
@@ -202,7 +213,7 @@ def ddtree_accept(target_logits, L: int, node_token, node_parent, n_rows, worksp
         out = Acceptance(torch.empty(R, **i32), torch.empty(R, L, **i32), torch.empty(R, L, **i32),
                          torch.empty(R, **i32), torch.empty(R, N, **i32))
     if workspace is None:
-        workspace = torch.empty(max(lib().ddtree_accept_workspace_bytes(R, B, V), 256), dtype=torch.uint8, device=dev)
+        workspace = _scratch(lib().ddtree_accept_workspace_bytes(R, B, V), dev, stream)
     _check(lib().ddtree_accept(
         target_logits.data_ptr(), _dtype_code(target_logits), target_logits.stride(1), R, B, V, L,
         node_token.data_ptr(), node_parent.data_ptr(), n_rows.data_ptr(), out.accept_len.data_ptr(),
@@ -228,7 +239,7 @@ def ddtree_accept_sampled(target_logits, L: int, node_token, node_parent, n_rows
         out = Acceptance(torch.empty(R, **i32), torch.empty(R, L, **i32), torch.empty(R, L, **i32),
                          torch.empty(R, **i32), torch.empty(R, N, **i32))
     if workspace is None:
-        workspace = torch.empty(max(lib().ddtree_accept_sampled_workspace_bytes(R, B, V), 256), dtype=torch.uint8, device=dev)
+        workspace = _scratch(lib().ddtree_accept_sampled_workspace_bytes(R, B, V), dev, stream)
     _check(lib().ddtree_accept_sampled(
         target_logits.data_ptr(), _dtype_code(target_logits), target_logits.stride(1), R, B, V, L,
         node_token.data_ptr(), node_parent.data_ptr(), n_rows.data_ptr(), float(temperature), row_uniform.data_ptr(),

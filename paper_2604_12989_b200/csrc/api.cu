@@ -247,6 +247,7 @@ static int fill_attn_args(const char* fn, AttnArgs& a, const void* q, const void
     a.q = q; a.k_cache = k_cache; a.v_cache = v_cache; a.k_tree = k_tree; a.v_tree = v_tree;
     a.cu_prefix = cu_prefix; a.anc_mask = anc_mask; a.n_rows = n_rows; a.out = out; a.lse = lse;
     a.R = R; a.B = B; a.N = B + 1; a.W = (B + 1 + 31) / 32; a.Hq = Hq; a.Hkv = Hkv; a.G = G; a.d = d;
+    if (!(scale >= 0.f) || !(scale <= 3.0e38f)) return fail(DDTREE_ERR_INVALID_ARG, "%s: softmax_scale must be positive and finite (0 = 1/sqrt(d))", fn);
     a.scale = scale != 0.f ? scale : 1.0f / sqrtf(static_cast<float>(d));
     a.max_prefix = max_p;
     a.total_prefix = cu_prefix_host[R];

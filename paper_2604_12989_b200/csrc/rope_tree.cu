@@ -1,5 +1,6 @@
 // Rotary positional encoding of the tree's query and key rows at the position ids ddtree_build assigned
-// ("position ids by tree depth so that the verifier applies the correct positional encoding", Section 4.4).
+// (Section 4.4: position ids follow the tree depth, so that every node is encoded at the position it would have
+// in its own branch).
 // Pair (j, j + d/2) of every head of row i is rotated by position_ids[i] * theta^(-2j/d) (half-split form).
 //
 // A pass of its own, in place, before the attention call rather than a step of the attention kernel's load
