@@ -44,10 +44,11 @@ def test_static_scratch_matches_workspace_variant_twice_in_a_row():
         want = dd.ddtree_accept(target, w.L, tree.node_token, tree.node_parent, tree.n_rows)
         out = empty_acceptance(w)
         torch.cuda.synchronize()
-        before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
+        counters = lambda: (torch.cuda.memory_stats()["allocation.all.allocated"], torch.cuda.memory_reserved())
+        before = counters()  # allocation requests served so far, bytes held from the driver
         got = dd.ddtree_accept_static_scratch(target, w.L, tree.node_token, tree.node_parent, tree.n_rows, out=out)
         torch.cuda.synchronize()
-        assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == before  # nothing was allocated
+        assert counters() == before  # the call asked torch's allocator for nothing, and nothing was reserved
         for name in ("accept_len", "accept_nodes", "accept_tokens", "bonus_token", "node_argmax"):
             assert torch.equal(getattr(got, name), getattr(want, name)), (seed, name)
         assert int(want.accept_len.max()) >= 1  # the walk did something
