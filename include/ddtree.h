@@ -200,6 +200,11 @@ int ddtree_accept(const void* target_logits, int dt, int64_t row_stride_elems,
  *   row_uniform   [R, B+1] uint32    device memory; entries of padding rows are not read
  * Outputs as for ddtree_accept; node_choice [R, B+1] (optional) receives the drawn token of every row,
  * padding rows -1.  A row whose logits have no finite maximum gets choice -1 (the walk stops there).
+ * The walk only consults the rows it stands on (the root and the accepted nodes: at most L + 1 per
+ * request).  With node_choice == NULL the call draws at those rows only: one cluster of CTAs per request
+ * follows the walk and reads each visited row once (vocabularies up to 458,000 tokens; larger ones, and
+ * calls that ask for node_choice, weigh every row in passes over all target logits).  The draw, and so every
+ * output, is the same either way.
  * V <= 2^22.  Errors as for ddtree_accept; temperature <= 0 or not finite -> DDTREE_ERR_INVALID_ARG.
  * ------------------------------------------------------------------------------------------ */
 size_t ddtree_accept_sampled_workspace_bytes(int R, int B, int V);

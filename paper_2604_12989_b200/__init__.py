@@ -223,10 +223,12 @@ def ddtree_accept(target_logits, L: int, node_token, node_parent, n_rows, worksp
 
 
 def ddtree_accept_sampled(target_logits, L: int, node_token, node_parent, n_rows, temperature: float, row_uniform,
-                          workspace=None, out: Optional[Acceptance] = None, stream=None) -> Acceptance:
+                          workspace=None, out: Optional[Acceptance] = None, stream=None, all_rows: bool = True) -> Acceptance:
     """ddtree_accept under the temperature-based decoding rule: the target's choice at a row is drawn from
     softmax(target_logits / temperature) with the row's 32-bit random input (row_uniform: [R, B+1], an int32
-    or uint32 CUDA tensor whose bit patterns are used).  `node_argmax` of the result holds the drawn tokens."""
+    or uint32 CUDA tensor whose bit patterns are used).  `node_argmax` of the result holds the drawn tokens of
+    every row; with all_rows=False the call draws only at the rows the walk stands on (much cheaper) and leaves
+    `node_argmax` untouched."""
     import torch
     R, N, V = target_logits.shape
     B = N - 1
@@ -244,7 +246,7 @@ def ddtree_accept_sampled(target_logits, L: int, node_token, node_parent, n_rows
         target_logits.data_ptr(), _dtype_code(target_logits), target_logits.stride(1), R, B, V, L,
         node_token.data_ptr(), node_parent.data_ptr(), n_rows.data_ptr(), float(temperature), row_uniform.data_ptr(),
         out.accept_len.data_ptr(), out.accept_nodes.data_ptr(), out.accept_tokens.data_ptr(), out.bonus_token.data_ptr(),
-        _ptr(out.node_argmax), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+        _ptr(out.node_argmax) if all_rows else None, workspace.data_ptr(), workspace.numel(), _stream(stream)))
     return out
 
 

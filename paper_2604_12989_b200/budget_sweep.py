@@ -91,7 +91,7 @@ def run(budgets, rounds, layers, prefix, seed=0, draft_boost0=5.0, draft_slope=0
             if temperature > 0:
                 uni = torch.randint(-2 ** 31, 2 ** 31 - 1, (1, w.N), generator=gen, device=dev, dtype=torch.int32)
                 acc = dd.ddtree_accept_sampled(target, w.L, tree.node_token, tree.node_parent, tree.n_rows, temperature, uni,
-                                               workspace=ws_a, out=acc)
+                                               workspace=ws_a, out=acc, all_rows=False)
             else:
                 acc = dd.ddtree_accept(target, w.L, tree.node_token, tree.node_parent, tree.n_rows, workspace=ws_a, out=acc)
             dd.ddtree_kv_compact(kt, vt, kc, vc, dst, acc.accept_len, acc.accept_nodes)

@@ -159,6 +159,13 @@ int ddtree_accept_sampled(const void* target_logits, int dt, int64_t row_stride_
     if (workspace_bytes < lay.total)
         return fail(DDTREE_ERR_WORKSPACE, "ddtree_accept_sampled: workspace %zu < required %zu bytes", workspace_bytes, lay.total);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (!node_choice && sampled_walk_fits(V)) {
+        // nobody asked for the choice at every row: draw only at the rows the walk stands on
+        const cudaError_t el = launch_sampled_walk(target_logits, dt, row_stride_elems, R, B + 1, V, L, n_rows, c, row_uniform,
+                                                   node_token, node_parent, accept_len, accept_nodes, accept_tokens, bonus_token, st);
+        if (el != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_accept_sampled: walk kernel: %s", cudaGetErrorString(el));
+        return DDTREE_OK;
+    }
     cudaError_t e = launch_row_argmax(target_logits, dt, row_stride_elems, R, B + 1, V, n_rows, lay.a, workspace, st);
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_accept_sampled: maximum pass: %s", cudaGetErrorString(e));
     e = launch_row_sample(target_logits, dt, row_stride_elems, R, B + 1, V, n_rows, c, row_uniform, lay, workspace, st);

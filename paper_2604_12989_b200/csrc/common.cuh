@@ -66,6 +66,14 @@ cudaError_t launch_row_sample(const void* logits, int dt, int64_t row_stride, in
                               float log2e_over_t, const uint32_t* row_uniform, const SampleLayout& lay, void* ws,
                               cudaStream_t st);
 
+// The sampled walk without the all-rows passes: one cluster of CTAs per request draws the target's choice only at the
+// rows the walk stands on (at most L + 1).  `sampled_walk_fits`: whether a row's slice fits a CTA's shared memory.
+bool sampled_walk_fits(int V);
+cudaError_t launch_sampled_walk(const void* logits, int dt, int64_t row_stride, int R, int N, int V, int L, const int32_t* n_rows,
+                                float log2e_over_t, const uint32_t* row_uniform, const int32_t* node_token,
+                                const int32_t* node_parent, int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
+                                int32_t* bonus_token, cudaStream_t st);
+
 // Rotary positional encoding of the tree's Q / K rows, in place (either pointer may be NULL).
 cudaError_t launch_rope_tree(void* q, void* k, const int32_t* position_ids, const int32_t* n_rows, int dt, int R, int N,
                              int Hq, int Hkv, int d, double log2_theta, cudaStream_t st);

@@ -10,6 +10,7 @@
 // All read each element once per pass with 16-byte loads; chunk partials are merged by the kernels in
 // tree_build.cu / accept_walk.cu.
 #include "common.cuh"
+#include <cooperative_groups.h>
 #include <math_constants.h>
 
 namespace ddtree {
@@ -359,6 +360,171 @@ row_sample_kernel(const T* __restrict__ logits, int64_t row_stride, int N, int V
     }
 }
 
+
+// ---- the sampled walk, lazily ----------------------------------------------------------------------------------
+// The walk only ever asks for the target's choice at the rows it stands on: the root, then one accepted node
+// per step, at most L + 1 rows of a request (Section 4.4).  Instead of weighing every row of every request,
+// a cluster of kWalkCtas CTAs per request follows the walk: at each visited row every CTA stages its slice of
+// the row's logits in shared memory (one read of the row), the CTAs exchange slice maxima and slice weight
+// sums through distributed shared memory, the CTA whose slice holds the threshold finds the token, and all of
+// them take the walk's step.  The draw is the one ddtree_accept_sampled defines (fixed-point weights relative
+// to the row maximum, threshold floor(total * k / 2^32), smallest token whose inclusive prefix sum exceeds
+// it): integer sums, so the partition into slices and threads does not matter.
+constexpr int kWalkCtas = 8;
+constexpr int kWalkThreads = 512;
+constexpr int kWalkWarps = kWalkThreads / 32;
+constexpr int kWalkMaxSlice = 56 * 1024;  // fp32 elements of one CTA's slice that fit its shared memory
+
+struct WalkShared {
+    float cmax;                          // this CTA's slice maximum (read by the other CTAs of the cluster)
+    unsigned long long csum;             // this CTA's slice weight sum
+    int ctok;                            // the drawn token, written by the CTA whose slice holds the threshold
+    float wmax[kWalkWarps];
+    unsigned long long wsum[kWalkWarps];
+    int found;
+    int token[kMaxN];
+    short parent[kMaxN];
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kWalkThreads, 1)
+sampled_walk_kernel(const T* __restrict__ logits, int64_t row_stride, int N, int V, int L, int slice,
+                    const int32_t* __restrict__ n_rows, float c, const uint32_t* __restrict__ row_uniform,
+                    const int32_t* __restrict__ node_token, const int32_t* __restrict__ node_parent,
+                    int32_t* __restrict__ accept_len, int32_t* __restrict__ accept_nodes,
+                    int32_t* __restrict__ accept_tokens, int32_t* __restrict__ bonus_token) {
+    namespace cg = cooperative_groups;
+    constexpr int VN = Vec16<T>::N;
+    extern __shared__ __align__(16) unsigned char walk_smem[];
+    WalkShared& sh = *reinterpret_cast<WalkShared*>(walk_smem);
+    float* xs = reinterpret_cast<float*>(walk_smem + ((sizeof(WalkShared) + 15) / 16) * 16);  // the staged slice, fp32
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = static_cast<int>(cluster.block_rank());
+    const int r = blockIdx.x / kWalkCtas, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_wait();
+    const int n = min(n_rows[r], N);
+    const size_t o = static_cast<size_t>(r) * N;
+    for (int row = tid; row < n; row += kWalkThreads) {
+        sh.token[row] = node_token[o + row];
+        sh.parent[row] = static_cast<short>(node_parent[o + row]);
+    }
+    const int begin = rank * slice, end = min(V, begin + slice);  // my tokens (begin is a multiple of 8)
+    const int count = max(0, end - begin);
+    const int per = ((slice + kWalkThreads - 1) / kWalkThreads) | 1;  // tokens per thread in the scan; odd: no bank conflicts
+    const WalkShared* peer[kWalkCtas];
+#pragma unroll
+    for (int k = 0; k < kWalkCtas; ++k) peer[k] = cluster.map_shared_rank(&sh, k);
+    __syncthreads();
+
+    int cur = 0, len = 0, tok = -1;
+    for (;;) {
+        // ---- 1. stage my slice of row `cur`, slice maximum ------------------------------------------------
+        const T* x = logits + static_cast<int64_t>(o + cur) * row_stride + begin;
+        float m = -CUDART_INF_F;
+        const int vec_count = (count / VN) * VN;
+        for (int i = tid * VN; i < vec_count; i += kWalkThreads * VN) {
+            float v[VN];
+            Vec16<T>::load(x + i, v);
+#pragma unroll
+            for (int e = 0; e < VN; ++e) { xs[i + e] = v[e]; m = fmaxf(m, v[e]); }
+        }
+        for (int i = vec_count + tid; i < count; i += kWalkThreads) {
+            const float v = Vec16<T>::scalar(x + i);
+            xs[i] = v;
+            m = fmaxf(m, v);
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, d));
+        if (lane == 0) sh.wmax[warp] = m;
+        __syncthreads();
+        if (tid == 0) {
+            float mm = sh.wmax[0];
+            for (int k = 1; k < kWalkWarps; ++k) mm = fmaxf(mm, sh.wmax[k]);
+            sh.cmax = mm;
+        }
+        cluster.sync();
+        float row_max = -CUDART_INF_F;
+#pragma unroll
+        for (int k = 0; k < kWalkCtas; ++k) row_max = fmaxf(row_max, peer[k]->cmax);
+
+        // ---- 2. weights of my slice: thread t owns tokens [t * per, (t + 1) * per) of it -----------------------
+        const int t0 = min(count, tid * per), t1 = min(count, t0 + per);
+        unsigned long long mine = 0;
+        for (int i = t0; i < t1; ++i) mine += sample_weight(xs[i], row_max, c);
+        unsigned long long incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned long long up = __shfl_up_sync(kFull, incl, d);
+            if (lane >= d) incl += up;
+        }
+        if (lane == 31) sh.wsum[warp] = incl;
+        __syncthreads();
+        unsigned long long before_me = 0, slice_total = 0;
+        for (int k = 0; k < kWalkWarps; ++k) {
+            if (k < warp) before_me += sh.wsum[k];
+            slice_total += sh.wsum[k];
+        }
+        incl += before_me;
+        if (tid == 0) { sh.csum = slice_total; sh.ctok = -1; }
+        cluster.sync();
+        unsigned long long total = 0, before_slice = 0;
+#pragma unroll
+        for (int k = 0; k < kWalkCtas; ++k) {
+            const unsigned long long sk = peer[k]->csum;
+            if (k < rank) before_slice += sk;
+            total += sk;
+        }
+
+        // ---- 3. the draw: the thread whose tokens hold the threshold names the token ---------------------------
+        if (total > 0) {  // else: no finite maximum in the row, nothing to draw from (token -1, the walk stops)
+            const unsigned long long u = row_uniform[o + cur];
+            const unsigned long long thr = (__umul64hi(total, u) << 32) | ((total * u) >> 32);  // floor(total * u / 2^32) < total
+            const unsigned long long lo = before_slice + (incl - mine), hi = before_slice + incl;
+            if (lo <= thr && thr < hi) {  // exactly one thread of the cluster
+                unsigned long long acc = lo;
+                int found = t1 - 1;
+                for (int i = t0; i < t1; ++i) {
+                    acc += sample_weight(xs[i], row_max, c);
+                    if (acc > thr) { found = i; break; }
+                }
+                sh.ctok = begin + found;
+            }
+        }
+        cluster.sync();
+        tok = -1;
+#pragma unroll
+        for (int k = 0; k < kWalkCtas; ++k) tok = max(tok, peer[k]->ctok);
+
+        // ---- 4. the walk's step (every CTA takes it; rank 0 writes) -------------------------------------------
+        if (len >= L || tok < 0) break;
+        if (tid == 0) sh.found = 0x7fffffff;
+        __syncthreads();
+        for (int j = cur + 1 + tid; j < n; j += kWalkThreads)   // children have larger rows; siblings carry distinct tokens
+            if (sh.parent[j] == cur && sh.token[j] == tok) atomicMin(&sh.found, j);
+        __syncthreads();
+        const int found = sh.found;
+        if (found == 0x7fffffff) break;
+        if (rank == 0 && tid == 0) {
+            accept_nodes[static_cast<size_t>(r) * L + len] = found;
+            accept_tokens[static_cast<size_t>(r) * L + len] = tok;
+        }
+        cur = found;
+        ++len;
+        __syncthreads();  // sh.found and the staged slice are rewritten in the next round
+    }
+    if (rank == 0) {
+        for (int k = len + tid; k < L; k += kWalkThreads) {
+            accept_nodes[static_cast<size_t>(r) * L + k] = -1;
+            accept_tokens[static_cast<size_t>(r) * L + k] = -1;
+        }
+        if (tid == 0) {
+            accept_len[r] = len;
+            bonus_token[r] = tok;
+        }
+    }
+    cluster.sync();  // no CTA leaves while a neighbour may still read its shared memory
+}
+
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 int pick_chunk(int64_t rows, int V, int lo, int hi) {
@@ -462,6 +628,46 @@ cudaError_t launch_row_sample(const void* logits, int dt, int64_t row_stride, in
     return launch_pdl(row_sample_kernel<__nv_bfloat16>, dim3(rows), dim3(kThreads), 0, st,
                       static_cast<const __nv_bfloat16*>(logits), row_stride, N, V, n_rows, lay.a.chunk_elems, lay.a.chunks,
                       log2e_over_t, pval, psum, row_uniform, token);
+}
+
+bool sampled_walk_fits(int V) { return (V + kWalkCtas - 1) / kWalkCtas <= kWalkMaxSlice - 8; }
+
+template <typename T>
+static cudaError_t launch_sampled_walk_t(const T* logits, int64_t row_stride, int R, int N, int V, int L, const int32_t* n_rows,
+                                         float c, const uint32_t* row_uniform, const int32_t* node_token, const int32_t* node_parent,
+                                         int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens, int32_t* bonus_token,
+                                         cudaStream_t st) {
+    const int slice = ((V + kWalkCtas - 1) / kWalkCtas + 7) / 8 * 8;  // slices start on 16-byte boundaries
+    const size_t smem = ((sizeof(WalkShared) + 15) / 16) * 16 + static_cast<size_t>(slice) * 4;
+    cudaError_t e = cudaFuncSetAttribute(sampled_walk_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(R) * kWalkCtas);
+    cfg.blockDim = dim3(kWalkThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kWalkCtas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, sampled_walk_kernel<T>, logits, row_stride, N, V, L, slice, n_rows, c, row_uniform, node_token,
+                              node_parent, accept_len, accept_nodes, accept_tokens, bonus_token);
+}
+
+cudaError_t launch_sampled_walk(const void* logits, int dt, int64_t row_stride, int R, int N, int V, int L, const int32_t* n_rows,
+                                float log2e_over_t, const uint32_t* row_uniform, const int32_t* node_token,
+                                const int32_t* node_parent, int32_t* accept_len, int32_t* accept_nodes, int32_t* accept_tokens,
+                                int32_t* bonus_token, cudaStream_t st) {
+    if (dt == DDTREE_F32)
+        return launch_sampled_walk_t(static_cast<const float*>(logits), row_stride, R, N, V, L, n_rows, log2e_over_t, row_uniform,
+                                     node_token, node_parent, accept_len, accept_nodes, accept_tokens, bonus_token, st);
+    return launch_sampled_walk_t(static_cast<const __nv_bfloat16*>(logits), row_stride, R, N, V, L, n_rows, log2e_over_t,
+                                 row_uniform, node_token, node_parent, accept_len, accept_nodes, accept_tokens, bonus_token, st);
 }
 
 }  // namespace ddtree

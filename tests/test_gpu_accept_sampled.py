@@ -51,6 +51,14 @@ def run_and_compare(w, trees, tl, T, ks):
         assert list(toks[:want.accept_len]) == want.tokens and (toks[want.accept_len:] == -1).all()
         assert int(acc.bonus_token[r]) == want.bonus_token
         lens.append(want.accept_len)
+    # the same call without node_choice: the library draws only at the rows the walk stands on (a cluster of
+    # CTAs per request follows the walk); every output must be the same
+    g2 = cases.Guard()
+    lazy = dd.ddtree_accept_sampled(t, w.L, tok, par, n_rows, T, u, workspace=ws, out=cases.guarded_acceptance(g2, w.R, w.L, w.N),
+                                    all_rows=False)
+    g2.check()
+    for name in ("accept_len", "accept_nodes", "accept_tokens", "bonus_token"):
+        assert torch.equal(getattr(lazy, name), getattr(acc, name)), name
     return lens
 
 
