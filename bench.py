@@ -39,7 +39,7 @@ NOMINAL = {"hbm_gbs": 8000.0, "tflops": 2250.0}  # the figures the benchmark spec names 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of tree_attention_bf16_kernel, from the ncu captures
 # summarised in profiles/tree_attention_bf16_config{1,2,4}.txt (None: no capture of that workload)
-NCU_TRAFFIC_BYTES = {1: None, 2: None, 4: None}
+NCU_TRAFFIC_BYTES = {1: 17746944, 2: 73499904, 4: 512054272}
 MIN_TIMED_SECONDS = 1.0
 
 
@@ -518,7 +518,7 @@ def measure_config(w, dev, args, rank, world, barrier, sampler, headline):
     for _ in range(max(3, args.warmup)):
         rb.graph.replay()
     torch.cuda.synchronize()
-    first, mean_ms, min_ms, blocks, t0, t1 = rb.time_graph(rb.graph, steps, MIN_TIMED_SECONDS, barrier)
+    first, mean_ms, min_ms, blocks, t0, t1 = rb.time_graph(rb.graph, steps, args.min_seconds, barrier)
     clocks = sampler.summary(t0, t1) if sampler else None
     ms_first = max_over_ranks(first, dev)
     ms_mean = max_over_ranks(mean_ms, dev)
@@ -527,7 +527,7 @@ def measure_config(w, dev, args, rank, world, barrier, sampler, headline):
     g_att = rb.attention_only_graph()
     for _ in range(3):
         g_att.replay()
-    a_first, a_mean, a_min, a_blocks, a0, a1 = rb.time_graph(g_att, max(1, steps // 2), MIN_TIMED_SECONDS, lambda: torch.cuda.synchronize())
+    a_first, a_mean, a_min, a_blocks, a0, a1 = rb.time_graph(g_att, max(1, steps // 2), args.min_seconds, lambda: torch.cuda.synchronize())
     att_call_ms = a_mean / w.layers
     att_region_s = a_mean * max(1, steps // 2) * a_blocks * 1e-3
     stage_ms = rb.stage_times()
@@ -753,6 +753,9 @@ def main():
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="0 = the greedy decoding rule (the benchmark's metric); > 0: the verifier walk samples the target's "
                          "choice at that temperature (ddtree_accept_sampled)")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="every workload's timed regions repeat their block of steps until this much device time has passed "
+                         "(0: one block; profiling runs)")
     ap.add_argument("--no-parity", action="store_true", help="skip the oracle comparison of every workload's outputs")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle (profiling runs)")
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
