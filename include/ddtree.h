@@ -238,6 +238,29 @@ int ddtree_rope_tree(void* q, void* k_tree, const int32_t* position_ids, const i
                      int dt, int R, int B, int Hq, int Hkv, int d, float rope_theta, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * ddtree_tree_attention_rope -- ddtree_tree_attention with the rotary positional encoding of Section 4.4
+ * (position ids by tree depth) applied inside the kernel's load path: q and k_tree are given UNROTATED and are
+ * not modified; every CTA rotates its query tile in shared memory once, before its first product, and the
+ * tiles of tree keys as they are staged (the cached keys were rotated when they were produced and are used as
+ * they are).  Same rule as ddtree_rope_tree: pair (j, j + d/2) of every head of row i is rotated by
+ * position_ids[r, i] * rope_theta^(-2j/d); angles in double precision, rotation in float32, rotated values
+ * rounded to bf16 before the products (as a separate ddtree_rope_tree pass would store them).  Equivalent to
+ * ddtree_rope_tree on copies of q and k_tree followed by ddtree_tree_attention.
+ *
+ * Arguments as for ddtree_tree_attention, plus position_ids [R, B+1] (as written by ddtree_build; a row sits
+ * at most 32 positions behind row 0 of its request) and rope_theta > 0.  dt must be DDTREE_BF16 (d = 128).
+ * The workspace size is ddtree_tree_attention_workspace_bytes(...).
+ * ------------------------------------------------------------------------------------------ */
+int ddtree_tree_attention_rope(const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* cu_prefix_host, const int32_t* cu_prefix,
+                               const void* k_tree, const void* v_tree,
+                               const uint32_t* anc_mask, const int32_t* n_rows,
+                               const int32_t* position_ids, float rope_theta,
+                               void* out, float* lse_or_null,
+                               int dt, int R, int B, int Hq, int Hkv, int d, float softmax_scale,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
  * ddtree_accept_static_scratch -- the paper has no counterpart; this is a packaging variant of
  * ddtree_accept for callers that cannot hand over a workspace.
  *

@@ -20,7 +20,7 @@ DDTREE_F32, DDTREE_BF16 = 0, 1
 EXPORTS = (
     "ddtree_status_string", "ddtree_last_error",
     "ddtree_build_workspace_bytes", "ddtree_build",
-    "ddtree_tree_attention_workspace_bytes", "ddtree_tree_attention",
+    "ddtree_tree_attention_workspace_bytes", "ddtree_tree_attention", "ddtree_tree_attention_rope",
     "ddtree_accept_workspace_bytes", "ddtree_accept", "ddtree_accept_static_scratch",
     "ddtree_accept_sampled_workspace_bytes", "ddtree_accept_sampled",
     "ddtree_kv_compact", "ddtree_rope_tree",
@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.ddtree_tree_attention_workspace_bytes.argtypes = [i32] * 6 + [vp]
         L.ddtree_tree_attention.restype = i32
         L.ddtree_tree_attention.argtypes = [vp] * 11 + [i32] * 6 + [f32, vp, sz, vp]
+        L.ddtree_tree_attention_rope.restype = i32
+        L.ddtree_tree_attention_rope.argtypes = [vp] * 10 + [f32, vp, vp] + [i32] * 6 + [f32, vp, sz, vp]
         L.ddtree_accept_workspace_bytes.restype = sz
         L.ddtree_accept_workspace_bytes.argtypes = [i32] * 3
         L.ddtree_accept.restype = i32
@@ -187,6 +189,32 @@ def ddtree_tree_attention(q, k_cache, v_cache, cu_prefix_host, cu_prefix, k_tree
         q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), ctypes.addressof(arr), cu_prefix.data_ptr(),
         k_tree.data_ptr(), v_tree.data_ptr(), anc_mask.data_ptr(), n_rows.data_ptr(), out.data_ptr(), _ptr(lse),
         code, R, B, Hq, Hkv, d, float(softmax_scale), workspace.data_ptr(), workspace.numel(), _stream(stream)))
+    return out
+
+
+def ddtree_tree_attention_rope(q, k_cache, v_cache, cu_prefix_host, cu_prefix, k_tree, v_tree, anc_mask, n_rows,
+                               position_ids, rope_theta: float, out=None, lse=None, softmax_scale: float = 0.0,
+                               workspace=None, stream=None):
+    """ddtree_tree_attention on UNROTATED bf16 q / k_tree: the rotary encoding at `position_ids` ([R, B+1], as
+    written by ddtree_build) is applied inside the kernel; q and k_tree are left as they are."""
+    import torch
+    R, N, Hq, d = q.shape
+    Hkv = k_tree.shape[2]
+    B = N - 1
+    for t in (q, k_cache, v_cache, k_tree, v_tree):
+        assert t.is_cuda and t.is_contiguous() and t.dtype == q.dtype
+    if out is None:
+        out = torch.zeros_like(q)
+    code = _dtype_code(q)
+    arr = (ctypes.c_int32 * (R + 1))(*[int(x) for x in cu_prefix_host])
+    if workspace is None:
+        need = lib().ddtree_tree_attention_workspace_bytes(R, B, Hq, Hkv, d, code, ctypes.addressof(arr))
+        workspace = _scratch(need, q.device, stream)
+    _check(lib().ddtree_tree_attention_rope(
+        q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), ctypes.addressof(arr), cu_prefix.data_ptr(),
+        k_tree.data_ptr(), v_tree.data_ptr(), anc_mask.data_ptr(), n_rows.data_ptr(), position_ids.data_ptr(),
+        float(rope_theta), out.data_ptr(), _ptr(lse), code, R, B, Hq, Hkv, d, float(softmax_scale),
+        workspace.data_ptr(), workspace.numel(), _stream(stream)))
     return out
 
 

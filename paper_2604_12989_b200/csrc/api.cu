@@ -293,6 +293,31 @@ int ddtree_tree_attention(const void* q, const void* k_cache, const void* v_cach
     return launch_tree_attention_bf16(a, cu_prefix_host, workspace, workspace_bytes, st);
 }
 
+int ddtree_tree_attention_rope(const void* q, const void* k_cache, const void* v_cache, const int32_t* cu_prefix_host,
+                               const int32_t* cu_prefix, const void* k_tree, const void* v_tree, const uint32_t* anc_mask,
+                               const int32_t* n_rows, const int32_t* position_ids, float rope_theta, void* out,
+                               float* lse_or_null, int dt, int R, int B, int Hq, int Hkv, int d, float softmax_scale,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    AttnArgs a;
+    int rc = fill_attn_args("ddtree_tree_attention_rope", a, q, k_cache, v_cache, cu_prefix_host, cu_prefix, k_tree, v_tree,
+                            anc_mask, n_rows, out, lse_or_null, dt, R, B, Hq, Hkv, d, softmax_scale, true);
+    if (rc) return rc;
+    if (dt != DDTREE_BF16)
+        return fail(DDTREE_ERR_UNSUPPORTED, "ddtree_tree_attention_rope: bf16 only (rotate fp32 rows with ddtree_rope_tree)");
+    if (!position_ids) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_tree_attention_rope: position_ids is NULL");
+    if (!(rope_theta > 0.f) || !(rope_theta <= 3.0e38f))
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_tree_attention_rope: rope_theta must be positive and finite");
+    a.rope = 1;
+    a.position_ids = position_ids;
+    a.rope_log2_theta = std::log2(static_cast<double>(rope_theta));
+    const size_t need = tree_attention_bf16_workspace(a, cu_prefix_host);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15u))
+        return fail(DDTREE_ERR_INVALID_ARG, "ddtree_tree_attention_rope: workspace is NULL or not 16-byte aligned");
+    if (workspace_bytes < need)
+        return fail(DDTREE_ERR_WORKSPACE, "ddtree_tree_attention_rope: workspace %zu < required %zu bytes", workspace_bytes, need);
+    return launch_tree_attention_bf16(a, cu_prefix_host, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
 // Scratch for ddtree_accept_static_scratch: lives in the library image, one copy per GPU that
 // loads it.  Host code must not pass `g_static_scratch` itself to a kernel: in host code that name
 // is only a handle for the runtime; the device address comes from cudaGetSymbolAddress.

@@ -89,6 +89,10 @@ struct AttnArgs {
     float scale;
     int max_prefix;     // host-side max over requests of P_r
     int64_t total_prefix;
+    // rotary variant (ddtree_tree_attention_rope): q and k_tree are rotated on their way into the products
+    int rope = 0;
+    const int32_t* position_ids = nullptr;
+    double rope_log2_theta = 0.0;
 };
 cudaError_t launch_tree_attention_f32(const AttnArgs& a, cudaStream_t st);
 

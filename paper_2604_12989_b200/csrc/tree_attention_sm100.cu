@@ -29,6 +29,7 @@
 #include <cuda_fp16.h>
 #include <math_constants.h>
 #include <algorithm>
+#include <cmath>
 #include <mutex>
 #include <type_traits>
 #include <unordered_map>
@@ -52,6 +53,7 @@ constexpr unsigned kFull = 0xffffffffu;
 constexpr int kMaxOrdered = 128;
 constexpr uint32_t kErrTimeout = 0x5101;
 constexpr uint32_t kErrAlign = 0x5102;
+constexpr int kRopeDepths = kMaxL + 1;  // a tree row sits at most kMaxL positions behind its root
 constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // 256 x 208 + 128 x 88 = 384 x 168 registers
 
 // ---- PTX wrappers --------------------------------------------------------------------------
@@ -237,6 +239,7 @@ struct Smem {
     uint8_t kv[kRing][kTileBytes];
     uint64_t q_full[2], kv_full[kRing], kv_free[kRing], v_fix[kRing];
     uint64_t s_full[2], p_half[2], p_ready[2], o_half[2], o_final[2];
+    uint64_t q_rot[2], k_rot[kRing];  // rotary variant: Q tile rotated by its row tile's threads, tree K tile by the relay warp
     uint32_t tmem_base;
     uint32_t abort;
 };
@@ -259,6 +262,10 @@ struct KernelParams {
     int units;        // CTAs per (request, KV head) = pairs * splits + tail * tail_splits
     int node0;        // the combine kernel covers nodes node0 .. N-1
     float scale_log2;
+    // rotary encoding applied on the way into the products (ddtree_tree_attention_rope): position ids of the tree rows
+    // and, per request and depth, cos / sin of position x frequency for the 64 frequency pairs of a head
+    const int32_t* position_ids;  // [R, N]
+    const float2* rope_table;     // [R, kRopeDepths, 64] (cos, sin), depth = position - position of the request's root
     // grid index -> request, longest prefix first (CTAs are dispatched in index order: the long ones must
     // not be left for the end); identity when the batch has more than kMaxOrdered requests
     int ordered;
@@ -772,7 +779,35 @@ __device__ __forceinline__ bool tile_visibility(uint32_t (&vis)[4], int t, int p
     return all_visible;
 }
 
-template <bool kTail>
+// Rotary encoding of one row of a staged Q or K tile (two 64-wide halves of 128 rows x 128 bytes, 16-byte chunks
+// swizzled with the row index): pair (j, j + 64) is rotated by the angle whose (cos, sin) is tab[j], in float32,
+// and rounded back to bf16 in place.
+__device__ __forceinline__ void rotate_row(uint8_t* tile, int row, const float2* __restrict__ tab) {
+#pragma unroll 2
+    for (int c = 0; c < 8; ++c) {
+        uint8_t* lo_p = tile + row * 128 + ((c ^ (row & 7)) << 4);
+        uint4 lo = *reinterpret_cast<const uint4*>(lo_p), hi = *reinterpret_cast<const uint4*>(lo_p + kHalfBytes);
+        __nv_bfloat16* xe = reinterpret_cast<__nv_bfloat16*>(&lo);
+        __nv_bfloat16* ye = reinterpret_cast<__nv_bfloat16*>(&hi);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float2 cs = __ldg(tab + c * 8 + e);
+            const float x = __bfloat162float(xe[e]), y = __bfloat162float(ye[e]);
+            xe[e] = __float2bfloat16_rn(x * cs.x - y * cs.y);
+            ye[e] = __float2bfloat16_rn(y * cs.x + x * cs.y);
+        }
+        *reinterpret_cast<uint4*>(lo_p) = lo;
+        *reinterpret_cast<uint4*>(lo_p + kHalfBytes) = hi;
+    }
+}
+// The table row of tree node `node` of request r (its depth = its position minus the root's).
+__device__ __forceinline__ const float2* rope_row(const KernelParams& p, int r, int node) {
+    const int32_t* pos = p.position_ids + static_cast<size_t>(r) * p.N;
+    const int depth = min(max(pos[node] - pos[0], 0), kRopeDepths - 1);
+    return p.rope_table + (static_cast<size_t>(r) * kRopeDepths + depth) * 64;
+}
+
+template <bool kTail, bool kRope>
 __global__ void __launch_bounds__(kThreads, 1)
 tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kc,
                            const __grid_constant__ CUtensorMap map_vc, const __grid_constant__ CUtensorMap map_kt,
@@ -844,7 +879,10 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             mbar_init(smem_u32(&sm.kv_full[s]), 1);
             mbar_init(smem_u32(&sm.kv_free[s]), 1);
             mbar_init(smem_u32(&sm.v_fix[s]), 1);
+            mbar_init(smem_u32(&sm.k_rot[s]), 1);
         }
+        mbar_init(smem_u32(&sm.q_rot[0]), kTile);
+        mbar_init(smem_u32(&sm.q_rot[1]), kTile);
         sm.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
@@ -897,6 +935,15 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                     const int first = keys_in_tile(t_begin + (u >> 1), prefix_tiles, P, n);
                     if (first < kTile) clear_v_rows(sm.kv[s], first, lane);
                     if (lane == 0) mbar_arrive(smem_u32(&sm.v_fix[s]));
+                } else if (kRope && t_begin + (u >> 1) >= prefix_tiles) {
+                    // a tile of this round's tree keys: rotate its rows to their positions (cached keys were
+                    // rotated when they were produced); rows past the tree are left as they are (masked anyway)
+                    const int node0 = (t_begin + (u >> 1) - prefix_tiles) * kTile;
+                    for (int row = lane; row < kTile; row += 32)
+                        if (node0 + row < n) rotate_row(sm.kv[s], row, rope_row(p, r, node0 + row));
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sm.k_rot[s]));
                 }
             }
         } else if (warp == kMmaWarp) {
@@ -939,14 +986,25 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             };
             auto wait_unit = [&](int u) { return wait_bar(&sm.kv_full[u % kRing], (u / kRing) & 1); };
             const int last_x = has_b ? 1 : 0;  // the row tile whose products release the K/V slots
-            bool ok = wait_bar(&sm.q_full[0], 0) && wait_unit(0);
+            uint32_t rot_phase = 0;  // rotary variant: per ring slot, parity of its next rotated tree K tile
+            // K tile of ring unit u staged (and, for a tile of tree keys in the rotary variant, rotated)
+            auto wait_k = [&](int u) {
+                bool good = wait_unit(u);
+                if (kRope && good && t_begin + (u >> 1) >= prefix_tiles) {
+                    const int s = u % kRing;
+                    good = wait_bar(&sm.k_rot[s], (rot_phase >> s) & 1);
+                    rot_phase ^= 1u << s;
+                }
+                return good;
+            };
+            bool ok = wait_bar(kRope ? &sm.q_rot[0] : &sm.q_full[0], 0) && wait_k(0);
             if (ok) {
                 tc_fence_after();
                 if (elect_one()) { issue_qk(0, 0); tc_commit(smem_u32(&sm.s_full[0])); if (!has_b) tc_commit(smem_u32(&sm.kv_free[0])); }
                 __syncwarp();
             }
             if (ok && has_b) {
-                ok = wait_bar(&sm.q_full[1], 0);
+                ok = wait_bar(kRope ? &sm.q_rot[1] : &sm.q_full[1], 0);
                 if (ok) {
                     tc_fence_after();
                     if (elect_one()) { issue_qk(1, 0); tc_commit(smem_u32(&sm.s_full[1])); tc_commit(smem_u32(&sm.kv_free[0])); }
@@ -960,7 +1018,7 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                     if (x == 0) {
                         // V_j staged and passed on by the clean-up warp (a slot holds K and V tiles in turn: every
                         // other use is a V tile), K_{j+1} staged: copies run far ahead, these rarely wait
-                        ok = wait_bar(&sm.v_fix[sv_slot], ((uv / kRing) >> 1) & 1) && (!more || wait_unit(uv + 1));
+                        ok = wait_bar(&sm.v_fix[sv_slot], ((uv / kRing) >> 1) & 1) && (!more || wait_k(uv + 1));
                         if (!ok) break;
                     }
                     // the probabilities arrive in two halves of 64 keys: the product over the first half runs
@@ -1006,6 +1064,13 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
             const uint32_t o_addr = lane_addr + kColO + x * kTile;
             float m_run = -CUDART_INF_F, l_run = 0.f;  // reference maximum (scaled log2 units; -inf: no key seen yet), sum
             bool ok = true;
+            if constexpr (kRope) {
+                // rotary variant: every thread rotates its own query row in the staged tile before the first product
+                ok = __all_sync(kFull, mbar_wait(smem_u32(&sm.q_full[x]), 0, abort_flag));
+                if (ok && valid) rotate_row(sm.q[x], row, rope_row(p, r, node));
+                fence_async_smem();
+                mbar_arrive(smem_u32(&sm.q_rot[x]));
+            }
             // A tile's scores come from tensor memory one half (64 columns) at a time: few registers are live (with
             // all 128 scores of a row in registers the compiler has no room to keep exponentials in flight), and
             // there are only two round trips per tile (a load in flight holds the warp back; the other row tile's
@@ -1199,6 +1264,28 @@ combine_kernel(const KernelParams p) {
     if (p.lse && lane == 0) p.lse[(static_cast<size_t>(r) * p.N + node) * p.Hq + h] = (M + log2f(l)) / kLog2e;
 }
 
+// Rotary variant: (cos, sin) of position x theta^(-2j/128) for every request, every depth a tree row can have and
+// the 64 frequency pairs of a head.  The angle is formed and reduced modulo 2 pi in double precision (positions
+// reach 10^5, where a float32 angle is off by 10^-2 rad), sine and cosine are taken in float32 on the reduced angle.
+struct RopeFreq64 {
+    double inv_freq[64];
+};
+__global__ void rope_table_kernel(const int32_t* __restrict__ position_ids, int N, float2* __restrict__ table,
+                                  const __grid_constant__ RopeFreq64 f) {
+    pdl_wait();
+    const int r = blockIdx.x;
+    const double pos0 = static_cast<double>(position_ids[static_cast<size_t>(r) * N]);  // the root's position
+    for (int i = threadIdx.x; i < kRopeDepths * 64; i += blockDim.x) {
+        const int depth = i >> 6, j = i & 63;
+        const double a = (pos0 + depth) * f.inv_freq[j];
+        const double turns = rint(a * 0.15915494309189535);
+        const double red = fma(-turns, 2.4492935982947064e-16, fma(-turns, 6.283185307179586, a));
+        float sn, cs;
+        sincosf(static_cast<float>(red), &sn, &cs);
+        table[(static_cast<size_t>(r) * kRopeDepths + depth) * 64 + j] = make_float2(cs, sn);
+    }
+}
+
 // A wait that nothing can satisfy: one thread initialises a barrier nobody arrives at, polls it `limit`
 // times, gives up and raises the time-out flag in the device status word, exactly as the attention
 // kernel's waits do.  The kernel returns normally.  (Self-test of the reporting path: see
@@ -1296,7 +1383,7 @@ struct Plan {
     int row_tiles, rows_pad;
     int full_tiles, pairs, tail;
     int splits, tail_splits, units;
-    size_t off_ml, total;
+    size_t off_ml, off_rope, total;
 };
 
 // How the rows and the KV range of a call are spread over CTAs.  A batch that fills the SMs more than once
@@ -1306,7 +1393,8 @@ Plan make_plan(const AttnArgs& a) {
     Plan pl;
     pl.row_tiles = (a.N * a.G + kTile - 1) / kTile;
     pl.rows_pad = pl.row_tiles * kTile;
-    pl.tail = (a.N * a.G - (pl.row_tiles - 1) * kTile <= kTailRows) ? 1 : 0;
+    // (the rotary variant runs a short last tile through the main path: one code path rotates)
+    pl.tail = (!a.rope && a.N * a.G - (pl.row_tiles - 1) * kTile <= kTailRows) ? 1 : 0;
     pl.full_tiles = pl.row_tiles - pl.tail;
     pl.pairs = (pl.full_tiles + 1) / 2;
     const int groups = a.R * a.Hkv;
@@ -1332,14 +1420,22 @@ Plan make_plan(const AttnArgs& a) {
     const int smax = std::max(pl.splits, pl.tail ? pl.tail_splits : 1);
     const size_t rows = static_cast<size_t>(smax) * a.R * a.Hkv * pl.rows_pad;
     pl.off_ml = (rows * kTile * 2 + 255) / 256 * 256;
-    pl.total = pl.off_ml + (rows * 8 + 255) / 256 * 256;
-    if (smax == 1) { pl.off_ml = 0; pl.total = 256; }
+    pl.off_rope = pl.off_ml + (rows * 8 + 255) / 256 * 256;
+    if (smax == 1) { pl.off_ml = 0; pl.off_rope = 0; }
+    pl.total = pl.off_rope + (a.rope ? static_cast<size_t>(a.R) * kRopeDepths * 64 * sizeof(float2) : 0);
+    if (pl.total < 256) pl.total = 256;
     return pl;
 }
 
 }  // namespace
 
-size_t tree_attention_bf16_workspace(const AttnArgs& a, const int32_t*) { return make_plan(a).total; }
+size_t tree_attention_bf16_workspace(const AttnArgs& a, const int32_t*) {
+    // one answer for ddtree_tree_attention and ddtree_tree_attention_rope (their plans differ in the short tile)
+    AttnArgs plain = a, rope = a;
+    plain.rope = 0;
+    rope.rope = 1;
+    return std::max(make_plan(plain).total, make_plan(rope).total);
+}
 
 int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host, void* ws, size_t, cudaStream_t st) {
     const Plan pl = make_plan(a);
@@ -1372,6 +1468,8 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
     // the combine kernel visits every row when the pairs are split, else only the short tile's rows
     p.node0 = pl.splits > 1 ? 0 : (pl.full_tiles * kTile) / a.G;
     p.scale_log2 = a.scale * kLog2e;
+    p.position_ids = a.position_ids;
+    p.rope_table = reinterpret_cast<const float2*>(static_cast<const char*>(ws) + pl.off_rope);
     p.ordered = 0;
     if (cu_prefix_host && a.R > 1 && a.R <= kMaxOrdered) {
         std::vector<int> idx(a.R);
@@ -1393,10 +1491,13 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
         cudaGetDevice(&dev);
         std::lock_guard<std::mutex> g(mu);
         if (dev < 0 || dev >= 64 || !done[dev]) {
-            cudaError_t e = cudaFuncSetAttribute(tree_attention_bf16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaError_t e = cudaFuncSetAttribute(tree_attention_bf16_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  static_cast<int>(smem_bytes));
             if (e == cudaSuccess)
-                e = cudaFuncSetAttribute(tree_attention_bf16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                e = cudaFuncSetAttribute(tree_attention_bf16_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem_bytes));
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(tree_attention_bf16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(smem_bytes));
             if (e != cudaSuccess)
                 return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: shared memory opt-in: %s", cudaGetErrorString(e));
@@ -1406,9 +1507,19 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
     const long long ctas = static_cast<long long>(a.R) * a.Hkv * pl.units;
     if (ctas > 0x7fffffffLL) return fail(DDTREE_ERR_UNSUPPORTED, "ddtree_tree_attention: grid too large");
     dim3 grid(static_cast<unsigned>(ctas));
-    cudaError_t e = pl.tail
-        ? launch_pdl(tree_attention_bf16_kernel<true>, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, mqt, p)
-        : launch_pdl(tree_attention_bf16_kernel<false>, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, mqt, p);
+    cudaError_t e = cudaSuccess;
+    if (a.rope) {
+        RopeFreq64 f;
+        for (int j = 0; j < 64; ++j) f.inv_freq[j] = std::exp2(-(2.0 * j / kTile) * a.rope_log2_theta);
+        e = launch_pdl(rope_table_kernel, dim3(a.R), dim3(256), 0, st, a.position_ids,  a.N,
+                       reinterpret_cast<float2*>(static_cast<char*>(ws) + pl.off_rope), f);
+        if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention_rope: table: %s", cudaGetErrorString(e));
+        e = launch_pdl(tree_attention_bf16_kernel<false, true>, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, mqt, p);
+    } else {
+        e = pl.tail
+            ? launch_pdl(tree_attention_bf16_kernel<true, false>, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, mqt, p)
+            : launch_pdl(tree_attention_bf16_kernel<false, false>, grid, dim3(kThreads), smem_bytes, st, mq, mkc, mvc, mkt, mvt, mqt, p);
+    }
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: launch: %s", cudaGetErrorString(e));
     if (pl.splits > 1 || (pl.tail && pl.tail_splits > 1)) {
         const long long tasks = static_cast<long long>(a.R) * (a.N - p.node0) * a.Hq;

@@ -107,3 +107,95 @@ def test_rope_argument_errors():
             dd.ddtree_rope_tree(q, None, pos, n_rows, theta)
     with pytest.raises(AssertionError):
         dd.ddtree_rope_tree(None, None, pos, n_rows, 1e6)
+
+
+# ---------------------------------------------------------------------------------------------
+# ddtree_tree_attention_rope: the same encoding applied inside the attention kernel's load path
+# ---------------------------------------------------------------------------------------------
+
+def fused_vs_oracle(w, trees, att, theta, softmax_scale=0.0):
+    """The fused call on unrotated rows against the oracle's attention over the oracle's rotated rows (rounded to
+    bf16 as the kernel rounds them before its products)."""
+    import paper_2604_12989_b200 as dd
+    q, kc, vc, kt, vt = (cases.to_torch(getattr(att, n), True) for n in ("q", "k_cache", "v_cache", "k_tree", "v_tree"))
+    q0, kt0 = q.clone(), kt.clone()
+    pos = torch.from_numpy(np.stack([t.position_ids for t in trees])).cuda()
+    n_rows = torch.tensor([t.n_rows for t in trees], dtype=torch.int32).cuda()
+    mask = torch.from_numpy(np.stack([t.mask for t in trees]).view(np.int32)).cuda()
+    cu = torch.from_numpy(att.cu_prefix).cuda()
+    lse = torch.zeros(w.R, w.N, w.Hq, dtype=torch.float32, device="cuda")
+    out = dd.ddtree_tree_attention_rope(q, kc, vc, att.cu_prefix.tolist(), cu, kt, vt, mask, n_rows, pos, theta, lse=lse,
+                                        softmax_scale=softmax_scale)
+    torch.cuda.synchronize()
+    dd.device_status()
+    assert torch.equal(q, q0) and torch.equal(kt, kt0)  # inputs are not modified
+    got = out.float().cpu().numpy().astype(np.float64)
+    worst = 0.0
+    for r in range(w.R):
+        n = trees[r].n_rows
+        lo, hi = att.cu_prefix[r], att.cu_prefix[r + 1]
+        qr = np.zeros_like(att.as_f64("q")[r])
+        kr = np.zeros_like(att.as_f64("k_tree")[r])
+        qr[:n] = wl.bf16_to_f64(wl.f32_to_bf16_bits(orc.rope(att.as_f64("q")[r, :n], trees[r].position_ids[:n], theta).astype(np.float32)))
+        kr[:n] = wl.bf16_to_f64(wl.f32_to_bf16_bits(orc.rope(att.as_f64("k_tree")[r, :n], trees[r].position_ids[:n], theta).astype(np.float32)))
+        kw = {} if softmax_scale == 0.0 else {"scale": softmax_scale}
+        ref, ref_lse = orc.tree_attention(qr, att.as_f64("k_cache")[lo:hi], att.as_f64("v_cache")[lo:hi], kr,
+                                          att.as_f64("v_tree")[r], trees[r].mask, n, **kw)
+        err = np.abs(got[r, :n] - ref) / (1 + np.abs(ref))
+        worst = max(worst, err.max())
+        assert err.max() <= 1e-2, f"request {r}: {err.max():.3e}"
+        np.testing.assert_allclose(lse[r, :n].cpu().numpy(), ref_lse, atol=2e-2, rtol=1e-2)
+        assert (got[r, n:] == 0).all()
+    return worst
+
+
+@pytest.mark.parametrize("R,B,Hq,Hkv,prefix", [
+    (1, 64, 8, 2, (700,)),            # split KV range, one tree tile, 4 rows left over (no short-tile path in this variant)
+    (2, 200, 4, 1, (260, 100000)),     # two tree tiles, a long-context position (angles need the double-precision reduction)
+    (3, 40, 16, 4, (0, 129, 5)),       # no cached context: every key tile is a rotated tree tile
+    (40, 31, 16, 4, None),             # a batch that fills the GPU: unsplit
+    (1, 1024, 16, 1, (300,)),          # the largest tree: nine tree tiles
+])
+def test_fused_rope_attention_equals_the_oracle_on_rotated_rows(R, B, Hq, Hkv, prefix):
+    if prefix is None:
+        prefix = tuple(int(x) for x in np.random.default_rng(3).integers(1, 400, R))
+    w, trees, att = build_case(R, B, Hq, Hkv, 128, "bf16", prefix)
+    fused_vs_oracle(w, trees, att, 1.0e6)
+
+
+def test_fused_rope_equals_the_separate_pass():
+    """ddtree_rope_tree on copies followed by ddtree_tree_attention, against the fused call: the same rotated
+    bf16 rows enter the same products, so the outputs agree to within the rounding of the rotation itself."""
+    import paper_2604_12989_b200 as dd
+    w, trees, att = build_case(2, 100, 8, 2, 128, "bf16", (900, 77))
+    theta = 1.0e4
+    q, kc, vc, kt, vt = (cases.to_torch(getattr(att, n), True) for n in ("q", "k_cache", "v_cache", "k_tree", "v_tree"))
+    pos = torch.from_numpy(np.stack([t.position_ids for t in trees])).cuda()
+    n_rows = torch.tensor([t.n_rows for t in trees], dtype=torch.int32).cuda()
+    mask = torch.from_numpy(np.stack([t.mask for t in trees]).view(np.int32)).cuda()
+    cu = torch.from_numpy(att.cu_prefix).cuda()
+    fused = dd.ddtree_tree_attention_rope(q, kc, vc, att.cu_prefix.tolist(), cu, kt, vt, mask, n_rows, pos, theta)
+    q2, kt2 = q.clone(), kt.clone()
+    dd.ddtree_rope_tree(q2, kt2, pos, n_rows, theta)
+    sep = dd.ddtree_tree_attention(q2, kc, vc, att.cu_prefix.tolist(), cu, kt2, vt, mask, n_rows)
+    torch.cuda.synchronize()
+    dd.device_status()
+    a, b = fused.float(), sep.float()
+    assert float(((a - b).abs() / (1 + b.abs())).max()) <= 4e-3
+
+
+def test_fused_rope_argument_errors():
+    import paper_2604_12989_b200 as dd
+    w, trees, att = build_case(1, 8, 2, 1, 128, "bf16", (3,))
+    q, kc, vc, kt, vt = (cases.to_torch(getattr(att, n), True) for n in ("q", "k_cache", "v_cache", "k_tree", "v_tree"))
+    pos = torch.from_numpy(trees[0].position_ids[None]).cuda()
+    n_rows = torch.tensor([trees[0].n_rows], dtype=torch.int32).cuda()
+    mask = torch.from_numpy(trees[0].mask[None].view(np.int32)).cuda()
+    cu = torch.from_numpy(att.cu_prefix).cuda()
+    for theta in (0.0, -1.0, float("inf")):
+        with pytest.raises(dd.DDTreeError):
+            dd.ddtree_tree_attention_rope(q, kc, vc, att.cu_prefix.tolist(), cu, kt, vt, mask, n_rows, pos, theta)
+    with pytest.raises(dd.DDTreeError) as e:  # fp32 has no fused variant
+        dd.ddtree_tree_attention_rope(q.float(), kc.float(), vc.float(), att.cu_prefix.tolist(), cu, kt.float(), vt.float(),
+                                      mask, n_rows, pos, 1e6)
+    assert e.value.status == 2
