@@ -122,6 +122,15 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// 32 contiguous bytes in one store: a full sector per request (with 16-byte stores of rows 256 bytes apart every
+// request fills half a sector and an SM moves 16 instead of 32 bytes per clock).  The address must be 32-byte aligned.
+__device__ __forceinline__ void st_global_256(void* p, const uint32_t (&v)[16], int o) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[o]), "r"(v[o + 1]), "r"(v[o + 2]),
+                 "r"(v[o + 3]), "r"(v[o + 4]), "r"(v[o + 5]), "r"(v[o + 6]), "r"(v[o + 7]) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory");
+}
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 // One lane of a converged warp (all 32 lanes must call this together).
 __device__ __forceinline__ bool elect_one() {
@@ -820,6 +829,34 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         return;
     }
 
+    // Barriers and descriptor prefetches touch nothing the previous kernel of the stream may still be writing: they
+    // run before the wait for it, and before the first sizes come back from global memory.
+    if (threadIdx.x == kProducerWarp * 32) {
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(smem_u32(&sm.q_full[x]), 1);
+            mbar_init(smem_u32(&sm.s_full[x]), 1);
+            mbar_init(smem_u32(&sm.p_half[x]), kTile);
+            mbar_init(smem_u32(&sm.p_ready[x]), kTile);
+            mbar_init(smem_u32(&sm.o_half[x]), 1);
+            mbar_init(smem_u32(&sm.o_final[x]), 1);
+            mbar_init(smem_u32(&sm.q_rot[x]), kTile);
+        }
+        for (int s = 0; s < kRing; ++s) {
+            mbar_init(smem_u32(&sm.kv_full[s]), 1);
+            mbar_init(smem_u32(&sm.kv_free[s]), 1);
+            mbar_init(smem_u32(&sm.v_fix[s]), 1);
+            mbar_init(smem_u32(&sm.k_rot[s]), 1);
+        }
+        sm.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    } else if (threadIdx.x == kProducerWarp * 32 + 1) {
+        prefetch_tensormap(&map_q);
+        prefetch_tensormap(&map_kc);
+        prefetch_tensormap(&map_vc);
+        prefetch_tensormap(&map_kt);
+        prefetch_tensormap(&map_vt);
+    }
     pdl_wait();               // everything read below may come from the previous kernel of the stream
     const int unit = blockIdx.x % p.units;
     const int kvh = (blockIdx.x / p.units) % p.Hkv;
@@ -866,40 +903,22 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
         for (int h = 0; h < 2; ++h)
             tma_load_3d(smem_u32(sm.kv[s]) + h * kHalfBytes, map, smem_u32(&sm.kv_full[s]), h * 64, kvh, row);
     };
-    if (warp == kProducerWarp && lane == 0) {
-        for (int x = 0; x < 2; ++x) {
-            mbar_init(smem_u32(&sm.q_full[x]), 1);
-            mbar_init(smem_u32(&sm.s_full[x]), 1);
-            mbar_init(smem_u32(&sm.p_half[x]), kTile);
-            mbar_init(smem_u32(&sm.p_ready[x]), kTile);
-            mbar_init(smem_u32(&sm.o_half[x]), 1);
-            mbar_init(smem_u32(&sm.o_final[x]), 1);
-        }
-        for (int s = 0; s < kRing; ++s) {
-            mbar_init(smem_u32(&sm.kv_full[s]), 1);
-            mbar_init(smem_u32(&sm.kv_free[s]), 1);
-            mbar_init(smem_u32(&sm.v_fix[s]), 1);
-            mbar_init(smem_u32(&sm.k_rot[s]), 1);
-        }
-        mbar_init(smem_u32(&sm.q_rot[0]), kTile);
-        mbar_init(smem_u32(&sm.q_rot[1]), kTile);
-        sm.abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        fence_async_smem();
+    if (warp == kProducerWarp) {
+        // the first copies leave from seven lanes at once (one lane issuing fourteen copies takes ~0.4 us): Q_A and
+        // the first K tile (the first product needs both), Q_B, then the rest of the ring
         const int nodes_per_tile = kTile / p.G;
-        // Q_A, then the first K tile (the first product needs both), then Q_B and the rest of the ring
-        mbar_expect_tx(smem_u32(&sm.q_full[0]), kTileBytes);
-        for (int h = 0; h < 2; ++h)
-            tma_load_4d(smem_u32(sm.q[0]) + h * kHalfBytes, &map_q, smem_u32(&sm.q_full[0]), h * 64, 0, kvh,
-                        r * p.N + rt0 * nodes_per_tile);
-        load_unit(issued++);
-        if (has_b) {
-            mbar_expect_tx(smem_u32(&sm.q_full[1]), kTileBytes);
+        if (lane == 0 || (lane == 2 && has_b)) {
+            const int x = lane >> 1;
+            mbar_expect_tx(smem_u32(&sm.q_full[x]), kTileBytes);
             for (int h = 0; h < 2; ++h)
-                tma_load_4d(smem_u32(sm.q[1]) + h * kHalfBytes, &map_q, smem_u32(&sm.q_full[1]), h * 64, 0, kvh,
-                            r * p.N + (rt0 + 1) * nodes_per_tile);
+                tma_load_4d(smem_u32(sm.q[x]) + h * kHalfBytes, &map_q, smem_u32(&sm.q_full[x]), h * 64, 0, kvh,
+                            r * p.N + (rt0 + x) * nodes_per_tile);
+        } else if (lane == 1) {
+            load_unit(0);
+        } else if (lane >= 3 && lane < 2 + kRing && lane - 2 < units_total) {
+            load_unit(lane - 2);
         }
-        for (; issued < units_total && issued < kRing; ++issued) load_unit(issued);
+        issued = min(kRing, units_total);
     }
     if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
@@ -1165,9 +1184,8 @@ tree_attention_bf16_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
                         }
                     }
                     if (valid) {
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            *reinterpret_cast<uint4*>(dst16 + c0 + 8 * u) = make_uint4(w16[4 * u], w16[4 * u + 1], w16[4 * u + 2], w16[4 * u + 3]);
+                        st_global_256(dst16 + c0, w16, 0);
+                        st_global_256(dst16 + c0 + 16, w16, 8);
                     }
                 }
                 if (valid) {
