@@ -333,6 +333,17 @@ int ddtree_device_status(void);
  * kernel does not trap, fault or spin without bound. */
 int ddtree_selftest_wait_timeout(void* cuda_stream);
 
+/* Which bf16 attention kernel ddtree_tree_attention launches (no counterpart in the paper; a tuning and
+ * test hook).  The library has two: one whose CTAs hold two 128-row tiles of a KV head (the throughput
+ * kernel: batches that fill the SMs, long KV ranges) and one whose CTAs hold a single row tile with two
+ * threads per row (the latency kernel: a batch whose row tiles leave SMs idle unless the KV range is cut
+ * into a few tiles per CTA).  path 0 (the default) lets a cost model choose per call from the shapes; 1
+ * forces the first, 2 the second wherever it applies (all CTAs resident at once, no rotary variant).
+ * Process-wide, takes effect at the next call; the workspace size ddtree_tree_attention_workspace_bytes
+ * reports covers every choice.  Both kernels give results within the same tolerance of each other, not
+ * bit-identical ones.  Returns DDTREE_OK, or DDTREE_ERR_INVALID_ARG for a path outside 0..2. */
+int ddtree_tree_attention_set_path(int path);
+
 #ifdef __cplusplus
 }
 #endif

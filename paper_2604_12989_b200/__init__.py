@@ -24,7 +24,7 @@ EXPORTS = (
     "ddtree_accept_workspace_bytes", "ddtree_accept", "ddtree_accept_static_scratch",
     "ddtree_accept_sampled_workspace_bytes", "ddtree_accept_sampled",
     "ddtree_kv_compact", "ddtree_rope_tree",
-    "ddtree_device_status", "ddtree_selftest_wait_timeout",
+    "ddtree_device_status", "ddtree_selftest_wait_timeout", "ddtree_tree_attention_set_path",
 )
 
 _lib = None
@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.ddtree_kv_compact.argtypes = [i32] * 7 + [vp] * 7 + [vp]
         L.ddtree_device_status.restype = i32
         L.ddtree_device_status.argtypes = []
+        L.ddtree_tree_attention_set_path.restype = i32
+        L.ddtree_tree_attention_set_path.argtypes = [i32]
         L.ddtree_selftest_wait_timeout.restype = i32
         L.ddtree_selftest_wait_timeout.argtypes = [vp]
         _lib = L
@@ -332,6 +334,11 @@ def ddtree_kv_compact(k_tree, v_tree, k_cache, v_cache, dst_row, accept_len, acc
     _check(lib().ddtree_kv_compact(R, N - 1, L, Hkv, d, _dtype_code(k_tree[0]), layers, arr(k_tree), arr(v_tree),
                                    arr(k_cache), arr(v_cache), dst_row.data_ptr(), accept_len.data_ptr(),
                                    accept_nodes.data_ptr(), _stream(stream)))
+
+
+def tree_attention_set_path(path: int) -> None:
+    """0: the library chooses the bf16 attention kernel per call; 1 / 2: force the two-row-tile / one-row-tile kernel."""
+    _check(lib().ddtree_tree_attention_set_path(int(path)))
 
 
 def selftest_wait_timeout(stream=None) -> None:

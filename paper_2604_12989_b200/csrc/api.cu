@@ -364,6 +364,12 @@ int ddtree_accept_static_scratch(const void* target_logits, int dt, int64_t row_
                          cuda_stream);
 }
 
+int ddtree_tree_attention_set_path(int path) {
+    if (path < 0 || path > 2) return fail(DDTREE_ERR_INVALID_ARG, "ddtree_tree_attention_set_path: path %d is not 0, 1 or 2", path);
+    tree_attention_set_path(path);
+    return DDTREE_OK;
+}
+
 int ddtree_selftest_wait_timeout(void* cuda_stream) {
     const cudaError_t e = launch_wait_timeout_selftest(4096u, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return fail(DDTREE_ERR_CUDA, "ddtree_selftest_wait_timeout: %s", cudaGetErrorString(e));

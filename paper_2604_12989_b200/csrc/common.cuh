@@ -111,6 +111,7 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
 uint32_t* device_status_word();
 // One-thread kernel whose bounded wait runs out after `limit` polls and raises the time-out flag.
 cudaError_t launch_wait_timeout_selftest(uint32_t limit, cudaStream_t st);
+void tree_attention_set_path(int path);
 
 // ---- programmatic dependent launch ---------------------------------------------------------------
 // Every kernel of this library is launched with programmatic stream serialisation: it may be scheduled

@@ -24,11 +24,9 @@
 // the request's last tile.  Each split writes its normalised rows (fp16) with their reference maximum
 // and sum; a combine kernel merges them by log-sum-exp.  Every wait is bounded: when one gives up, the
 // CTA raises a flag in the device status word, drains its copies and leaves without touching its outputs.
-#include "common.cuh"
-#include <cuda.h>
-#include <cuda_fp16.h>
-#include <math_constants.h>
+#include "sm100_attention.cuh"
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <mutex>
 #include <type_traits>
@@ -37,211 +35,14 @@
 
 namespace ddtree {
 namespace {
+using namespace sm100;
 
-constexpr int kTile = 128;            // rows per row tile, keys per KV tile, head dim
 constexpr int kRing = 5;              // K/V tiles in flight: K_j in slot 2j % 5, V_j in slot (2j+1) % 5
 constexpr int kProducerWarp = 8, kMmaWarp = 9, kFixWarp = 10;
 constexpr int kThreads = 384;         // warps 0-3 / 4-7: softmax A / B; 8: producer; 9: MMA; 10: V clean-up; 11: idle
-constexpr uint32_t kHalfBytes = 128 * 64 * 2;      // one 64-wide half of a 128x128 bf16 tile
-constexpr uint32_t kTileBytes = 2 * kHalfBytes;
-constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0;         // S_X at column 128 X; P_X (bf16 pairs) in its first 64 columns
 constexpr uint32_t kColO = 256;       // O_X at column 256 + 128 X
-constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr unsigned kFull = 0xffffffffu;
-constexpr int kMaxOrdered = 128;
-constexpr uint32_t kErrTimeout = 0x5101;
-constexpr uint32_t kErrAlign = 0x5102;
-constexpr int kRopeDepths = kMaxL + 1;  // a tree row sits at most kMaxL positions behind its root
 constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // 256 x 208 + 128 x 88 = 384 x 168 registers
-
-// ---- PTX wrappers --------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Non-blocking test of a phase.  try_wait may park the thread for a while and costs a couple of
-// hundred cycles even when the phase has long completed; test_wait answers at once, so every wait
-// starts with it and several barriers can be tested back to back.
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false when it gave up (or another thread of the CTA already did).
-__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t limit) {
-    if (mbar_test(bar, parity)) return true;
-    for (uint32_t i = 0; i < limit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 32) {
-            __nanosleep(64);
-            if ((i & 255u) == 0 && *abort_flag) return false;
-        }
-    }
-    *abort_flag = 1;
-    return false;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
-    return mbar_wait_limit(bar, parity, abort_flag, kSpinLimit);
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// 32 contiguous bytes in one store: a full sector per request (with 16-byte stores of rows 256 bytes apart every
-// request fills half a sector and an SM moves 16 instead of 32 bytes per clock).  The address must be 32-byte aligned.
-__device__ __forceinline__ void st_global_256(void* p, const uint32_t (&v)[16], int o) {
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[o]), "r"(v[o + 1]), "r"(v[o + 2]),
-                 "r"(v[o + 3]), "r"(v[o + 4]), "r"(v[o + 5]), "r"(v[o + 6]), "r"(v[o + 7]) : "memory");
-}
-__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory");
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-// One lane of a converged warp (all 32 lanes must call this together).
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile(
-        "{\n\t.reg .pred P1;\n\t.reg .b32 r;\n\t"
-        "elect.sync r|P1, 0xffffffff;\n\t"
-        "selp.b32 %0, 1, 0, P1;\n\t}"
-        : "=r"(pred));
-    return pred != 0;
-}
-// Register budget of the calling warp group (all four warps of it execute this together).
-template <int kRegs> __device__ __forceinline__ void regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs)); }
-template <int kRegs> __device__ __forceinline__ void regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs)); }
-
-// D[tmem] (+)= A[smem desc] * B[smem desc].  The accumulate flag is a template argument and the
-// operands are "base + constant": one thread issues every MMA of the CTA, and anything beyond a
-// handful of scalar instructions per MMA makes that thread, not the tensor pipe, the bottleneck.
-template <bool kAccumulate>
-__device__ __forceinline__ void umma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc) {
-    if (kAccumulate)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                     ::"r"(d), "l"(a), "l"(b), "r"(idesc) : "memory");
-    else
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                     ::"r"(d), "l"(a), "l"(b), "r"(idesc) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem desc]
-template <bool kAccumulate>
-__device__ __forceinline__ void umma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc) {
-    if (kAccumulate)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-                     ::"r"(d), "r"(a), "l"(b), "r"(idesc) : "memory");
-    else
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
-                     "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-                     ::"r"(d), "r"(a), "l"(b), "r"(idesc) : "memory");
-}
-
-#define DDTREE_R32(a, o) \
-    "=r"(a[o + 0]), "=r"(a[o + 1]), "=r"(a[o + 2]), "=r"(a[o + 3]), "=r"(a[o + 4]), "=r"(a[o + 5]), "=r"(a[o + 6]),     \
-    "=r"(a[o + 7]), "=r"(a[o + 8]), "=r"(a[o + 9]), "=r"(a[o + 10]), "=r"(a[o + 11]), "=r"(a[o + 12]), "=r"(a[o + 13]), \
-    "=r"(a[o + 14]), "=r"(a[o + 15]), "=r"(a[o + 16]), "=r"(a[o + 17]), "=r"(a[o + 18]), "=r"(a[o + 19]),               \
-    "=r"(a[o + 20]), "=r"(a[o + 21]), "=r"(a[o + 22]), "=r"(a[o + 23]), "=r"(a[o + 24]), "=r"(a[o + 25]),               \
-    "=r"(a[o + 26]), "=r"(a[o + 27]), "=r"(a[o + 28]), "=r"(a[o + 29]), "=r"(a[o + 30]), "=r"(a[o + 31])
-#define DDTREE_W32(a, o) \
-    "r"(a[o + 0]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]), "r"(a[o + 5]), "r"(a[o + 6]),     \
-    "r"(a[o + 7]), "r"(a[o + 8]), "r"(a[o + 9]), "r"(a[o + 10]), "r"(a[o + 11]), "r"(a[o + 12]), "r"(a[o + 13]), \
-    "r"(a[o + 14]), "r"(a[o + 15]), "r"(a[o + 16]), "r"(a[o + 17]), "r"(a[o + 18]), "r"(a[o + 19]),             \
-    "r"(a[o + 20]), "r"(a[o + 21]), "r"(a[o + 22]), "r"(a[o + 23]), "r"(a[o + 24]), "r"(a[o + 25]),             \
-    "r"(a[o + 26]), "r"(a[o + 27]), "r"(a[o + 28]), "r"(a[o + 29]), "r"(a[o + 30]), "r"(a[o + 31])
-#define DDTREE_L32 \
-    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "   \
-    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}"
-#define DDTREE_S32 \
-    "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "  \
-    "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32}"
-
-// 32 consecutive columns of this thread's TMEM lane -> v[o .. o+31]
-#define TMEM_LD32(v, o, taddr) \
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 " DDTREE_L32 ", [%32];" : DDTREE_R32(v, o) : "r"(taddr))
-#define TMEM_ST32(taddr, v, o) \
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], " DDTREE_S32 ";" ::"r"(taddr), DDTREE_W32(v, o) : "memory")
-// 64 consecutive columns of this thread's TMEM lane -> v[0 .. 63] (one round trip: a load in flight holds the
-// warp's following instructions back, so fewer, wider loads are cheaper than several narrow ones)
-__device__ __forceinline__ void tmem_ld64(uint32_t (&v)[64], uint32_t taddr) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31]), "=r"(v[32]), "=r"(v[33]), "=r"(v[34]), "=r"(v[35]), "=r"(v[36]), "=r"(v[37]), "=r"(v[38]), "=r"(v[39]), "=r"(v[40]), "=r"(v[41]), "=r"(v[42]), "=r"(v[43]), "=r"(v[44]), "=r"(v[45]), "=r"(v[46]), "=r"(v[47]), "=r"(v[48]), "=r"(v[49]), "=r"(v[50]), "=r"(v[51]), "=r"(v[52]), "=r"(v[53]), "=r"(v[54]), "=r"(v[55]), "=r"(v[56]), "=r"(v[57]), "=r"(v[58]), "=r"(v[59]), "=r"(v[60]), "=r"(v[61]), "=r"(v[62]), "=r"(v[63])
-                 : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// 16 consecutive columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_ld16(uint32_t (&v)[16], uint32_t taddr) {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-                 : "r"(taddr));
-}
-// Named barriers of the short-tile path: id 1 + g over the 128 threads of key group g (plain and with an
-// OR vote), id 3 over both groups.
-__device__ __forceinline__ void bar_keys(int g) { asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory"); }
-__device__ __forceinline__ bool bar_keys_or(int g, bool x) {
-    uint32_t r;
-    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %2, 0;\n\tbar.red.or.pred p, %1, 128, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                 : "=r"(r) : "r"(1 + g), "r"(static_cast<uint32_t>(x)) : "memory");
-    return r != 0;
-}
-__device__ __forceinline__ void bar_all_keys() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
-
-// Shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart.
-//   K-major operand (Q, K): rows of 64 bf16 (128 bytes); the leading-dimension field is unused.
-//   MN-major operand (V):   rows are keys (the contraction index), 64 head-dim elements per row;
-//                           `lbo_bytes` is the distance between the two 64-wide head-dim halves.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((addr & 0x3ffffu) >> 4);
-    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3fffu) << 16;
-    d |= static_cast<uint64_t>(1024u >> 4) << 32;
-    d |= 1ull << 46;  // descriptor version of this architecture
-    d |= 2ull << 61;  // 128-byte swizzle
-    return d;
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n.
-__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) |
-           (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTile >> 4) << 24);
-}
 
 struct Smem {
     uint8_t q[2][kTileBytes];        // row tiles A and B
@@ -253,103 +54,6 @@ struct Smem {
     uint32_t abort;
 };
 
-struct KernelParams {
-    const int32_t* cu_prefix;
-    const uint32_t* anc_mask;
-    const int32_t* n_rows;
-    __nv_bfloat16* out;
-    float* lse;
-    __half* part_o;  // [S, R, Hkv, rows_pad, 128]: each split's O divided by its own sum, fp16
-    float2* part_ml; // [S, R, Hkv, rows_pad] (reference max in log2 units, sum)
-    uint32_t* status;
-    int R, N, W, Hq, Hkv, G, rows_pad;
-    int full_tiles;   // 128-row tiles handled in pairs by the CTAs of the main path
-    int pairs;        // ceil(full_tiles / 2)
-    int splits;       // KV splits of a pair
-    int tail;         // 1: the last 128-row tile (index full_tiles) is a short tile with a CTA of its own
-    int tail_splits;  // KV splits of the short tile
-    int units;        // CTAs per (request, KV head) = pairs * splits + tail * tail_splits
-    int node0;        // the combine kernel covers nodes node0 .. N-1
-    float scale_log2;
-    // rotary encoding applied on the way into the products (ddtree_tree_attention_rope): position ids of the tree rows
-    // and, per request and depth, cos / sin of position x frequency for the 64 frequency pairs of a head
-    const int32_t* position_ids;  // [R, N]
-    const float2* rope_table;     // [R, kRopeDepths, 64] (cos, sin), depth = position - position of the request's root
-    // grid index -> request, longest prefix first (CTAs are dispatched in index order: the long ones must
-    // not be left for the end); identity when the batch has more than kMaxOrdered requests
-    int ordered;
-    uint16_t order[kMaxOrdered];
-};
-
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// Two non-negative floats -> packed bf16 pair (low half = a), round to nearest even.
-__device__ __forceinline__ uint32_t pack_cvt(float a, float b) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
-    return r;
-}
-
-// Exponentials of the 64 scores of half a tile relative to the reference m_use, packed to bf16 pairs
-// (pk[c] = keys 2c, 2c+1 of the half, c < 32); returns their sum.
-__device__ __forceinline__ float exp_pack_64(const uint32_t (&x)[64], uint32_t (&pk)[32], float scale_log2, float m_use) {
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-#pragma unroll
-    for (int c = 0; c < 64; c += 4) {
-        const float e0 = ex2(fmaf(__uint_as_float(x[c]), scale_log2, -m_use));
-        const float e1 = ex2(fmaf(__uint_as_float(x[c + 1]), scale_log2, -m_use));
-        const float e2 = ex2(fmaf(__uint_as_float(x[c + 2]), scale_log2, -m_use));
-        const float e3 = ex2(fmaf(__uint_as_float(x[c + 3]), scale_log2, -m_use));
-        s0 += e0; s1 += e1; s2 += e2; s3 += e3;
-        pk[c >> 1] = pack_cvt(e0, e1);
-        pk[(c >> 1) + 1] = pack_cvt(e2, e3);
-    }
-    return (s0 + s1) + (s2 + s3);
-}
-
-__device__ __forceinline__ float max_64(const uint32_t (&x)[64]) {
-    float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-#pragma unroll
-    for (int c = 0; c < 64; c += 8)
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-            mx4[k] = max3(mx4[k], __uint_as_float(x[c + 2 * k]), __uint_as_float(x[c + 2 * k + 1]));
-    return fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]);
-}
-
-// Replace the scores of invisible keys by -inf: bit c of `word` tells whether key o + c is visible to this row.
-template <int kN>
-__device__ __forceinline__ void mask32(uint32_t (&sv)[kN], int o, uint32_t word) {
-#pragma unroll
-    for (int c = 0; c < 32; ++c)
-        if (!((word >> c) & 1u)) sv[o + c] = 0xff800000u;
-}
-
-// Number of keys of KV tile t (absolute index within the request) that any row may see: the rows of a
-// staged V tile from there on belong to another request, to padding or to nobody.
-__device__ __forceinline__ int keys_in_tile(int t, int prefix_tiles, int P, int n) {
-    return t < prefix_tiles ? min(kTile, P - t * kTile) : min(kTile, n - (t - prefix_tiles) * kTile);
-}
-// Zero rows [first, 128) of a staged V tile (both 64-wide halves; the 128-byte swizzle permutes 16-byte
-// chunks inside a row only).  Whole warp; the writes are made visible to the tensor pipe.
-__device__ __forceinline__ void clear_v_rows(uint8_t* tile, int first, int lane) {
-    const int chunks = (kTile - first) * 16;
-    for (int i = lane; i < chunks; i += 32) {
-        const int row = first + (i >> 4), c = i & 15;
-        *reinterpret_cast<uint4*>(tile + (c >> 3) * kHalfBytes + row * 128 + (c & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
-    }
-    fence_async_smem();
-    __syncwarp();
-}
 
 // ---- short last row tile ----------------------------------------------------------------------
 // A tree of B = 2^k nodes plus the root leaves G rows over for a last row tile of their own; run
@@ -1399,18 +1103,26 @@ constexpr int kSMs = 148;
 
 struct Plan {
     int row_tiles, rows_pad;
+    int halves;  // 1: one row tile per CTA (tree_attention_sm100_halves.cu), `splits` KV splits for every row tile
     int full_tiles, pairs, tail;
     int splits, tail_splits, units;
     size_t off_ml, off_rope, total;
 };
 
+std::atomic<int> g_path{0};  // 0: chosen by the cost model, 1: two row tiles per CTA, 2: one row tile per CTA
+
 // How the rows and the KV range of a call are spread over CTAs.  A batch that fills the SMs more than once
-// runs unsplit.  Otherwise every CTA is resident at once, and the KV range is split so that the pairs' CTAs
-// (~2800 cycles per KV tile) and the short tile's CTAs (~1250 cycles per tile) finish together.
-Plan make_plan(const AttnArgs& a) {
+// runs unsplit, two row tiles per CTA.  Otherwise every CTA is resident at once and the KV range is split so
+// that all CTAs finish together; the costs below (cycles, from device time stamps of layers whose K/V come
+// from HBM) are: a CTA of row-tile pairs 15600 + 4100 per KV tile, a short-tile CTA 24000 + 1400 per tile, a
+// CTA of one row tile 10000 + 2000 per tile.  With few tiles per CTA the fixed terms decide, and one row tile
+// per CTA reaches the same number of resident CTAs with half the splits (half the partial rows to write and
+// to merge).
+Plan make_plan(const AttnArgs& a, int path) {
     Plan pl;
     pl.row_tiles = (a.N * a.G + kTile - 1) / kTile;
     pl.rows_pad = pl.row_tiles * kTile;
+    pl.halves = 0;
     // (the rotary variant runs a short last tile through the main path: one code path rotates)
     pl.tail = (!a.rope && a.N * a.G - (pl.row_tiles - 1) * kTile <= kTailRows) ? 1 : 0;
     pl.full_tiles = pl.row_tiles - pl.tail;
@@ -1427,14 +1139,27 @@ Plan make_plan(const AttnArgs& a) {
         for (int s = 1; s <= (pl.pairs ? s_cap : 1); ++s) {
             for (int t = 1; t <= (pl.tail ? t_cap : 1); ++t) {
                 if (pl.pairs * s + pl.tail * t > budget) break;
-                const double cf = pl.pairs ? 9000.0 + 2800.0 * ((max_tiles + s - 1) / s) + (s > 1 ? 400.0 * s : 0.0) : 0.0;
-                const double ct = pl.tail ? 7000.0 + 1250.0 * ((max_tiles + t - 1) / t) : 0.0;
+                const double cf = pl.pairs ? 15600.0 + 4100.0 * ((max_tiles + s - 1) / s) : 0.0;
+                const double ct = pl.tail ? 24000.0 + 1400.0 * ((max_tiles + t - 1) / t) : 0.0;
                 const double cost = std::max(cf, ct) + 1.0 * (pl.pairs * s + pl.tail * t);  // ties: fewer CTAs
                 if (cost < best) { best = cost; pl.splits = s; pl.tail_splits = t; }
             }
         }
+        // one row tile per CTA instead?
+        if (!a.rope && path != 1 && groups * pl.row_tiles <= kSMs) {
+            const int s = std::max(1, std::min(std::min(32, kSMs / (groups * pl.row_tiles)), (max_tiles + 1) / 2));
+            const double ch = 10000.0 + 2000.0 * ((max_tiles + s - 1) / s);
+            if (path == 2 || ch < 0.92 * best) {
+                pl.halves = 1;
+                pl.tail = 0;
+                pl.full_tiles = pl.row_tiles;
+                pl.pairs = 0;
+                pl.splits = s;
+                pl.tail_splits = 1;
+            }
+        }
     }
-    pl.units = pl.pairs * pl.splits + pl.tail * pl.tail_splits;
+    pl.units = pl.halves ? pl.row_tiles * pl.splits : pl.pairs * pl.splits + pl.tail * pl.tail_splits;
     const int smax = std::max(pl.splits, pl.tail ? pl.tail_splits : 1);
     const size_t rows = static_cast<size_t>(smax) * a.R * a.Hkv * pl.rows_pad;
     pl.off_ml = (rows * kTile * 2 + 255) / 256 * 256;
@@ -1449,14 +1174,17 @@ Plan make_plan(const AttnArgs& a) {
 
 size_t tree_attention_bf16_workspace(const AttnArgs& a, const int32_t*) {
     // one answer for ddtree_tree_attention and ddtree_tree_attention_rope (their plans differ in the short tile)
+    // and whichever kernel the cost model or ddtree_tree_attention_set_path picks at launch time
     AttnArgs plain = a, rope = a;
     plain.rope = 0;
     rope.rope = 1;
-    return std::max(make_plan(plain).total, make_plan(rope).total);
+    return std::max(make_plan(rope, 1).total, std::max(make_plan(plain, 1).total, make_plan(plain, 2).total));
 }
 
+void tree_attention_set_path(int path) { g_path.store(path < 0 || path > 2 ? 0 : path, std::memory_order_relaxed); }
+
 int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host, void* ws, size_t, cudaStream_t st) {
-    const Plan pl = make_plan(a);
+    const Plan pl = make_plan(a, g_path.load(std::memory_order_relaxed));
     CUtensorMap mq, mkc, mvc, mkt, mvt, mqt;
     const uint64_t tree_rows = static_cast<uint64_t>(a.R) * a.N;
     int rc = get_map(&mq, a.q, 4, a.G, a.Hkv, tree_rows, a.G, kTile / a.G);
@@ -1517,6 +1245,7 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
             if (e == cudaSuccess)
                 e = cudaFuncSetAttribute(tree_attention_bf16_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          static_cast<int>(smem_bytes));
+            if (e == cudaSuccess) e = tree_attention_halves_opt_in();
             if (e != cudaSuccess)
                 return fail(DDTREE_ERR_CUDA, "ddtree_tree_attention: shared memory opt-in: %s", cudaGetErrorString(e));
             if (dev >= 0 && dev < 64) done[dev] = true;
@@ -1526,7 +1255,9 @@ int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host,
     if (ctas > 0x7fffffffLL) return fail(DDTREE_ERR_UNSUPPORTED, "ddtree_tree_attention: grid too large");
     dim3 grid(static_cast<unsigned>(ctas));
     cudaError_t e = cudaSuccess;
-    if (a.rope) {
+    if (pl.halves) {
+        e = launch_tree_attention_halves(dim3(pl.splits, a.Hkv * pl.row_tiles, a.R), mq, mkc, mvc, mkt, mvt, p, st);
+    } else if (a.rope) {
         RopeFreq64 f;
         for (int j = 0; j < 64; ++j) f.inv_freq[j] = std::exp2(-(2.0 * j / kTile) * a.rope_log2_theta);
         e = launch_pdl(rope_table_kernel, dim3(a.R), dim3(256), 0, st, a.position_ids,  a.N,

@@ -12,6 +12,16 @@ pytestmark = pytest.mark.gpu
 TOL = {"f32": 1e-4, "bf16": 1e-2}
 
 
+@pytest.fixture(params=["two_row_tiles", "one_row_tile"])
+def kernel_path(request):
+    """The library has two bf16 kernels and normally picks one per call from the shapes; tests that take this
+    fixture run once with each forced (a forced choice that does not apply to a shape falls back to the other)."""
+    import paper_2604_12989_b200 as dd
+    dd.tree_attention_set_path(1 if request.param == "two_row_tiles" else 2)
+    yield request.param
+    dd.tree_attention_set_path(0)
+
+
 def gpu_attention(w, att, trees, with_lse=True):
     import paper_2604_12989_b200 as dd
     bf = w.dtype == "bf16"
@@ -114,14 +124,14 @@ def bf16_case(R, B, Hq, Hkv, prefix_lens, K=4, L=8, seed=0, sentinel=False):
 
 
 @pytest.mark.parametrize("P", [0, 1, 7, 127, 128, 129, 300])
-def test_bf16_short_prefixes_and_sentinel_values(P):
+def test_bf16_short_prefixes_and_sentinel_values(P, kernel_path):
     w, att, trees = bf16_case(2, 70, 8, 2, (P, P + 5 if P else 0), sentinel=True)
     out, lse = gpu_attention(w, att, trees)
     compare(w, att, trees, out, lse)
 
 
 @pytest.mark.parametrize("profile", ["growing", "exploding", "shrinking"])
-def test_bf16_scores_that_outgrow_the_reference_maximum(profile):
+def test_bf16_scores_that_outgrow_the_reference_maximum(profile, kernel_path):
     # The kernel exponentiates a tile against the reference maximum it already has and looks at the
     # exact maximum only when a row sum comes near overflow.  Keys whose scale changes from one
     # 128-key tile to the next force that path: "growing" lifts the scores by ~2^30 per tile (row
@@ -137,13 +147,13 @@ def test_bf16_scores_that_outgrow_the_reference_maximum(profile):
 
 
 @pytest.mark.parametrize("G,Hkv", [(1, 2), (2, 2), (4, 1), (8, 1), (16, 1)])
-def test_bf16_group_sizes(G, Hkv):
+def test_bf16_group_sizes(G, Hkv, kernel_path):
     w, att, trees = bf16_case(1, 40, G * Hkv, Hkv, (200,), seed=G)
     out, lse = gpu_attention(w, att, trees)
     compare(w, att, trees, out, lse)
 
 
-def test_bf16_two_tree_tiles_and_heap_that_ran_empty():
+def test_bf16_two_tree_tiles_and_heap_that_ran_empty(kernel_path):
     # B = 200: tree keys span two 128-key tiles; second request has K = 1 chain (n_rows = 9 << B+1)
     w, att, trees = bf16_case(2, 200, 4, 1, (260, 3), K=4, L=8, seed=3)
     chain = orc.build(wl.drafter_logits(w, 1, "peak", 3), 1, w.B, 0, 3)
@@ -247,6 +257,15 @@ def test_bf16_full_size_workloads(cfg, heads_full, n_random):
     print(f"config {cfg}: worst scaled error {worst:.3e}")
 
 
+@pytest.mark.parametrize("cfg", [1, 2])
+def test_bf16_full_size_one_request_on_either_kernel(cfg, kernel_path):
+    """Workloads 1 and 2 (one request: every CTA resident at once, the KV range split) on each of the two kernels."""
+    w = wl.WORKLOADS[cfg]
+    att, trees = make_case(w, "peak", seed=3)
+    out, lse = gpu_attention(w, att, trees)
+    compare(w, att, trees, out, lse, sampled_pairs(w, trees, (7,), 24, 10 + cfg))
+
+
 def test_bf16_first_call_of_a_fresh_process():
     """The first launch of a process runs with cold instruction caches and unusual warp timing; a
     missed wait inside the kernel shows up there first.  Two-tile, unsplit case in a child process."""
@@ -265,7 +284,7 @@ def test_bf16_first_call_of_a_fresh_process():
     assert res.returncode == 0 and "fresh-process ok" in res.stdout, res.stdout + res.stderr
 
 
-def test_bf16_largest_tree_and_custom_scale():
+def test_bf16_largest_tree_and_custom_scale(kernel_path):
     """B = 1024 (1025 rows, 33 mask words, nine 128-key tree tiles), empty prefix, 16 query heads per KV
     head, a caller-chosen softmax scale and no lse output."""
     import paper_2604_12989_b200 as dd
@@ -292,7 +311,7 @@ def test_bf16_largest_tree_and_custom_scale():
         assert err.max() <= 1e-2, (i, h, err.max())
 
 
-def test_bf16_batch_with_an_empty_prefix_and_a_root_only_tree():
+def test_bf16_batch_with_an_empty_prefix_and_a_root_only_tree(kernel_path):
     """Request 0 has no cached context, request 2's tree is the root alone (n_rows = 1)."""
     w = wl.small_workload(R=3, L=6, V=900, K=3, B=37, Hq=8, Hkv=2, d=128, dtype="bf16", prefix_lens=(0, 700, 130), index=42)
     att, trees = make_case(w)
@@ -324,7 +343,7 @@ def test_bf16_workspace_too_small_is_refused():
 
 
 @pytest.mark.parametrize("seed", range(14))
-def test_bf16_random_shapes(seed):
+def test_bf16_random_shapes(seed, kernel_path):
     """Random small problems: batch size, budget, group size, prefix lengths (zero, a few keys, ragged
     ends of a 128-key tile, several tiles so that the KV range is split) and trees smaller than the
     budget, all rows against the oracle."""
@@ -344,7 +363,7 @@ def test_bf16_random_shapes(seed):
         assert (out[r, trees[r].n_rows:] == 0).all()  # rows past the tree are left alone
 
 
-def test_bf16_padding_inputs_may_hold_nan():
+def test_bf16_padding_inputs_may_hold_nan(kernel_path):
     """Rows of the inputs that the call must ignore are filled with NaN bit patterns: tree rows >= n_rows of
     q, k_tree and v_tree (one request's tree is smaller than the budget), and spare cache rows behind the
     last request's prefix.  Masked probabilities are zero, but the value rows of a masked key still travel
@@ -387,7 +406,7 @@ def test_bf16_padding_inputs_may_hold_nan():
         compare(w, att, trees, got, lse.cpu().numpy())
 
 
-def test_bf16_long_trains_of_launches_stay_identical():
+def test_bf16_long_trains_of_launches_stay_identical(kernel_path):
     """Hundreds of back-to-back launches on the large-budget workload's shapes, rotating over input sets larger
     than L2 so that the copies' arrival order varies: every launch must give bit for bit what the first launch
     on the same inputs gave, and no device-side wait may give up.  (A warp that watched only every other phase
