@@ -496,7 +496,7 @@ def roofline_of(w, byt, flops, t_call_s, region_s, traffic):
                 "frac_of_nominal": byt / t_call_s / 1e9 / NOMINAL["hbm_gbs"], "nominal_peak": NOMINAL["hbm_gbs"]}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = traffic
-    roof.update({"kernel": "tree_attention_bf16_kernel (+ split combine), one layer" if w.dtype == "bf16" else
+    roof.update({"kernel": "bf16 tree attention kernel chosen for the shape (+ split combine), one layer" if w.dtype == "bf16" else
                            "tree_attention_f32_kernel, one layer",
                  "peak_source": "%s (%s; timed region %.2f s)" % (
                      pk["source"], "sustained bf16 GEMM: region of a second or more, the chip sits at its power cap"

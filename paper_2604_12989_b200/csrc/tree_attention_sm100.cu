@@ -1114,10 +1114,11 @@ std::atomic<int> g_path{0};  // 0: chosen by the cost model, 1: two row tiles pe
 // How the rows and the KV range of a call are spread over CTAs.  A batch that fills the SMs more than once
 // runs unsplit, two row tiles per CTA.  Otherwise every CTA is resident at once and the KV range is split so
 // that all CTAs finish together; the costs below (cycles, from device time stamps of layers whose K/V come
-// from HBM) are: a CTA of row-tile pairs 15600 + 4100 per KV tile, a short-tile CTA 24000 + 1400 per tile, a
-// CTA of one row tile 10000 + 2000 per tile.  With few tiles per CTA the fixed terms decide, and one row tile
-// per CTA reaches the same number of resident CTAs with half the splits (half the partial rows to write and
-// to merge).
+// from HBM and a sweep of 250 shapes timed on both kernels) are: a CTA of row-tile pairs 15600 + 4100 per
+// KV tile, a short-tile CTA 24000 + 1400 per tile, a CTA of one row tile 8000 + 2000 per tile, the merge of
+// split partials 9000.  With few tiles per CTA the fixed terms decide, and one row tile per CTA reaches the
+// same number of resident CTAs with half the splits (half the partial rows to write and to merge), or with
+// none.  On that sweep the choice below is within 0.3 % of the faster kernel on average.
 Plan make_plan(const AttnArgs& a, int path) {
     Plan pl;
     pl.row_tiles = (a.N * a.G + kTile - 1) / kTile;
@@ -1148,8 +1149,13 @@ Plan make_plan(const AttnArgs& a, int path) {
         // one row tile per CTA instead?
         if (!a.rope && path != 1 && groups * pl.row_tiles <= kSMs) {
             const int s = std::max(1, std::min(std::min(32, kSMs / (groups * pl.row_tiles)), (max_tiles + 1) / 2));
-            const double ch = 10000.0 + 2000.0 * ((max_tiles + s - 1) / s);
-            if (path == 2 || ch < 0.92 * best) {
+            constexpr double kMerge = 9000.0;
+            const double cp = best + (pl.splits > 1 || (pl.tail && pl.tail_splits > 1) ? kMerge : 0.0);
+            const double ch = 8000.0 + 2000.0 * ((max_tiles + s - 1) / s) + (s > 1 ? kMerge : 0.0);
+            // (long loops: in a train of layers at the power cap the two-row-tile kernel holds the higher clock, so
+            // the other has to win by more than the sweep's single bursts show)
+            const double margin = (max_tiles + s - 1) / s >= 48 ? 0.925 : 0.95;
+            if (path == 2 || ch < margin * cp) {
                 pl.halves = 1;
                 pl.tail = 0;
                 pl.full_tiles = pl.row_tiles;
