@@ -39,7 +39,7 @@ NOMINAL = {"hbm_gbs": 8000.0, "tflops": 2250.0}  # the figures the benchmark spec names 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of tree_attention_bf16_kernel, from the ncu captures
 # summarised in profiles/tree_attention_bf16_config{1,2,4}.txt (None: no capture of that workload)
-NCU_TRAFFIC_BYTES = {1: 17746944, 2: 73499904, 4: 512054272}
+NCU_TRAFFIC_BYTES = {1: 17665024, 2: 73499904, 3: 392809216, 4: 512054272}
 MIN_TIMED_SECONDS = 1.0
 
 
@@ -748,7 +748,8 @@ def main():
     ap.add_argument("--config", type=int, default=HEADLINE_CONFIG,
                     help="headline workload (4 = the 70B-shaped long-context request, the largest that fits one GPU)")
     ap.add_argument("--configs", default="0,1,2,3,4", help="workloads of the per_config block (comma separated)")
-    ap.add_argument("--variant", default="lit", choices=wl.VARIANTS)
+    ap.add_argument("--variant", default="peak", choices=wl.VARIANTS,
+                    help="input recipe: `peak` gives accepted paths of several tokens, `lit` (the boost as written) accepts nothing")
     ap.add_argument("--layers", type=int, default=0, help="override the headline workload's layer count (profiling small cases only)")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="0 = the greedy decoding rule (the benchmark's metric); > 0: the verifier walk samples the target's "
