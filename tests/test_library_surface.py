@@ -83,3 +83,17 @@ def test_validation_without_gpu(lib):
     assert rope(q=None, k=None) == 1
     assert rope(dt=5) == 1
     assert lib.ddtree_rope_tree(p, p, None, p, 1, 1, 8, 4, 2, 128, 1e6, None) == 1   # no position ids
+
+
+def test_attention_kernel_choice_hook(lib):
+    """ddtree_tree_attention_set_path takes 0, 1 or 2 and refuses anything else; the workspace query does not
+    depend on it (it covers every kernel the call may pick)."""
+    cu = (ctypes.c_int32 * 2)(0, 4096)
+    sizes = []
+    for path in (0, 1, 2, 0):
+        assert lib.ddtree_tree_attention_set_path(path) == 0
+        sizes.append(lib.ddtree_tree_attention_workspace_bytes(1, 64, 32, 8, 128, 1, cu))
+    assert len(set(sizes)) == 1 and sizes[0] > 0
+    for bad in (-1, 3, 100):
+        assert lib.ddtree_tree_attention_set_path(bad) == 1
+    assert b"path" in lib.ddtree_last_error()
