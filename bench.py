@@ -340,7 +340,8 @@ class RoundBench:
         self.ws_att = torch.empty(max(256, dd.tree_attention_workspace_bytes(w.R, w.B, w.Hq, w.Hkv, w.d, 1 if bf else 0,
                                                                              self.cu_host)), **u8)
         self.acc = self.accept_call(self.target)
-        self.attn_kernels = 2 if (bf and self.ws_att.numel() > 256) else 1  # split-KV adds the combine kernel
+        # kernels per attention call, as the library plans it for these shapes (a split KV range adds the merge kernel)
+        self.attn_kernels = dd.tree_attention_kernel_count(w.R, w.B, w.Hq, w.Hkv, w.d, 1 if bf else 0, self.cu_host)
         self.launches_per_round = 2 + self.attn_kernels * w.layers + (1 if T > 0 else 2)
         self.stream = torch.cuda.Stream(device=dev)
         with torch.cuda.stream(self.stream):

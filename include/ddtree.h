@@ -344,6 +344,11 @@ int ddtree_selftest_wait_timeout(void* cuda_stream);
  * bit-identical ones.  Returns DDTREE_OK, or DDTREE_ERR_INVALID_ARG for a path outside 0..2. */
 int ddtree_tree_attention_set_path(int path);
 
+/* How many kernels of this library one ddtree_tree_attention call with these shapes launches under the current
+ * path setting: 1, or 2 when the KV range is split and a merge kernel follows (no counterpart in the paper; for
+ * launch accounting in benchmarks).  Arguments as for ddtree_tree_attention_workspace_bytes; 0 if they are invalid. */
+int ddtree_tree_attention_kernel_count(int R, int B, int Hq, int Hkv, int d, int dt, const int32_t* cu_prefix_host);
+
 #ifdef __cplusplus
 }
 #endif

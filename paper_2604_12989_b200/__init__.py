@@ -24,7 +24,7 @@ EXPORTS = (
     "ddtree_accept_workspace_bytes", "ddtree_accept", "ddtree_accept_static_scratch",
     "ddtree_accept_sampled_workspace_bytes", "ddtree_accept_sampled",
     "ddtree_kv_compact", "ddtree_rope_tree",
-    "ddtree_device_status", "ddtree_selftest_wait_timeout", "ddtree_tree_attention_set_path",
+    "ddtree_device_status", "ddtree_selftest_wait_timeout", "ddtree_tree_attention_set_path", "ddtree_tree_attention_kernel_count",
 )
 
 _lib = None
@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.ddtree_kv_compact.argtypes = [i32] * 7 + [vp] * 7 + [vp]
         L.ddtree_device_status.restype = i32
         L.ddtree_device_status.argtypes = []
+        L.ddtree_tree_attention_kernel_count.restype = i32
+        L.ddtree_tree_attention_kernel_count.argtypes = [i32] * 6 + [vp]
         L.ddtree_tree_attention_set_path.restype = i32
         L.ddtree_tree_attention_set_path.argtypes = [i32]
         L.ddtree_selftest_wait_timeout.restype = i32
@@ -167,6 +169,12 @@ def ddtree_build(drafter_logits, K: int, B: int, root_token, prefix_len, workspa
 def tree_attention_workspace_bytes(R, B, Hq, Hkv, d, dtype_code, cu_prefix_host) -> int:
     arr = (ctypes.c_int32 * (R + 1))(*[int(x) for x in cu_prefix_host])
     return lib().ddtree_tree_attention_workspace_bytes(R, B, Hq, Hkv, d, dtype_code, ctypes.addressof(arr))
+
+
+def tree_attention_kernel_count(R, B, Hq, Hkv, d, dtype_code, cu_prefix_host) -> int:
+    """Kernels one ddtree_tree_attention call with these shapes launches (1, or 2 with a split merge)."""
+    arr = (ctypes.c_int32 * (R + 1))(*[int(x) for x in cu_prefix_host])
+    return lib().ddtree_tree_attention_kernel_count(R, B, Hq, Hkv, d, dtype_code, ctypes.addressof(arr))
 
 
 def ddtree_tree_attention(q, k_cache, v_cache, cu_prefix_host, cu_prefix, k_tree, v_tree, anc_mask, n_rows,

@@ -271,6 +271,14 @@ size_t ddtree_tree_attention_workspace_bytes(int R, int B, int Hq, int Hkv, int 
     return tree_attention_bf16_workspace(a, cu_prefix_host);
 }
 
+int ddtree_tree_attention_kernel_count(int R, int B, int Hq, int Hkv, int d, int dt, const int32_t* cu_prefix_host) {
+    AttnArgs a;
+    if (fill_attn_args("ddtree_tree_attention_kernel_count", a, nullptr, nullptr, nullptr, cu_prefix_host, nullptr,
+                       nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, dt, R, B, Hq, Hkv, d, 0.f, false))
+        return 0;
+    return dt == DDTREE_F32 ? 1 : tree_attention_bf16_kernels(a);
+}
+
 int ddtree_tree_attention(const void* q, const void* k_cache, const void* v_cache, const int32_t* cu_prefix_host,
                           const int32_t* cu_prefix, const void* k_tree, const void* v_tree, const uint32_t* anc_mask,
                           const int32_t* n_rows, void* out, float* lse_or_null, int dt, int R, int B, int Hq, int Hkv,

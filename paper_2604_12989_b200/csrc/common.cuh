@@ -112,6 +112,8 @@ uint32_t* device_status_word();
 // One-thread kernel whose bounded wait runs out after `limit` polls and raises the time-out flag.
 cudaError_t launch_wait_timeout_selftest(uint32_t limit, cudaStream_t st);
 void tree_attention_set_path(int path);
+// kernels one bf16 attention call launches for these shapes (attention, + split merge, + rotary table)
+int tree_attention_bf16_kernels(const AttnArgs& a);
 
 // ---- programmatic dependent launch ---------------------------------------------------------------
 // Every kernel of this library is launched with programmatic stream serialisation: it may be scheduled

@@ -1187,6 +1187,11 @@ size_t tree_attention_bf16_workspace(const AttnArgs& a, const int32_t*) {
     return std::max(make_plan(rope, 1).total, std::max(make_plan(plain, 1).total, make_plan(plain, 2).total));
 }
 
+int tree_attention_bf16_kernels(const AttnArgs& a) {
+    const Plan pl = make_plan(a, g_path.load(std::memory_order_relaxed));
+    return 1 + ((pl.splits > 1 || (pl.tail && pl.tail_splits > 1)) ? 1 : 0) + (a.rope ? 1 : 0);
+}
+
 void tree_attention_set_path(int path) { g_path.store(path < 0 || path > 2 ? 0 : path, std::memory_order_relaxed); }
 
 int launch_tree_attention_bf16(const AttnArgs& a, const int32_t* cu_prefix_host, void* ws, size_t, cudaStream_t st) {

@@ -97,3 +97,14 @@ def test_attention_kernel_choice_hook(lib):
     for bad in (-1, 3, 100):
         assert lib.ddtree_tree_attention_set_path(bad) == 1
     assert b"path" in lib.ddtree_last_error()
+
+
+def test_attention_kernel_count(lib):
+    """One kernel when the rows fill the GPU (no KV split), two when a single request's KV range is split; fp32: one."""
+    lib.ddtree_tree_attention_set_path(0)
+    one = (ctypes.c_int32 * 2)(0, 4096)
+    assert lib.ddtree_tree_attention_kernel_count(1, 64, 32, 8, 128, 1, one) == 2
+    assert lib.ddtree_tree_attention_kernel_count(1, 16, 4, 1, 64, 0, one) == 1
+    many = (ctypes.c_int32 * 65)(*[512 * i for i in range(65)])
+    assert lib.ddtree_tree_attention_kernel_count(64, 128, 32, 8, 128, 1, many) == 1
+    assert lib.ddtree_tree_attention_kernel_count(1, 64, 32, 7, 128, 1, one) == 0  # Hq not a multiple of Hkv
