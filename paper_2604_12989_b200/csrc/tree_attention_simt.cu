@@ -87,14 +87,23 @@ tree_attention_f32_kernel(const float* __restrict__ q, const float* __restrict__
         m = m_new;
 #pragma unroll
         for (int e = 0; e < E; ++e) acc[e] *= alpha;
-        unsigned todo = any;
-        while (todo) {
-            const int src = __ffs(todo) - 1;
-            todo &= todo - 1;
-            const float pj = __shfl_sync(kFull, p, src);
-            const float* vrow = vbase + static_cast<size_t>(src) * Hkv * D;
+        // value rows of the visible keys, eight at a time: their loads leave together (a row that is not visible is
+        // not read at all: it may lie outside the request, or hold anything)
+        for (int s0 = 0; s0 < 32; s0 += 8) {
+            if (!((any >> s0) & 0xffu)) continue;  // warp-uniform
+            float pj[8], vv[8][E];
 #pragma unroll
-            for (int e = 0; e < E; ++e) acc[e] = fmaf(pj, __ldg(vrow + e * 32 + lane), acc[e]);
+            for (int u = 0; u < 8; ++u) {
+                const bool on = (any >> (s0 + u)) & 1u;
+                pj[u] = __shfl_sync(kFull, p, s0 + u);
+                const float* vrow = vbase + static_cast<size_t>(s0 + u) * Hkv * D;
+#pragma unroll
+                for (int e = 0; e < E; ++e) vv[u][e] = on ? __ldg(vrow + e * 32 + lane) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[e] = fmaf(pj[u], vv[u][e], acc[e]);
         }
     }
     float* orow = out + ((static_cast<size_t>(r) * N + i) * Hq + h) * D;
